@@ -1,0 +1,347 @@
+/*
+ * CPU oracle for the SCOPE sparse-attention layer.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, single-threaded restatement of what the paper defines, one
+ * attention head at a time, used to check the CUDA library and as the timed CPU
+ * baseline.  It shares no code with the CUDA path and must never be called from
+ * it.  Every stored real is fp32; every accumulation is fp64 and rounded once.
+ * Decisions that turn reals into integers (nearest centroid, Top-p count) are
+ * taken in fp64.
+ *
+ * Functions follow the paper's steps in its own order:
+ *   scope_oracle_kmeans      KMeans(X, C) of Algorithm 1 line 1 and Algorithm 2
+ *                            line 3; nearest centroid as in Eq. 3, mean as in Eq. 2
+ *   scope_oracle_lut         score table P_m of Eq. 5
+ *   scope_oracle_scores_row  indexed sum of Eq. 6 (before the 1/sqrt(d) factor)
+ *   scope_oracle_topp_row    descending ranking and Top-p count of Eq. 7
+ *   scope_oracle_khead       Eq. 8, Eq. 9 and the counts r_c of Eq. 10
+ *   scope_oracle_key_set     the set S_c of Eq. 10
+ *   scope_oracle_attn_row    one output row of Eq. 11
+ *   scope_oracle_dense_row   one output row of Eq. 1
+ *
+ * Readings taken where the paper is silent (also listed in the design notes):
+ * evenly strided initial centroids, a fixed number of Lloyd iterations, squared
+ * Euclidean distance for queries and keys alike, lowest index wins a tie, an
+ * empty cluster keeps its centroid, the returned assignment is the one of the
+ * last assignment step and the returned centroids are the means of exactly those
+ * members, equal proxy logits are ranked by ascending key index, softmax is
+ * evaluated with the row maximum subtracted.
+ *
+ * Parity pins: every function here is pinned by tests/test_oracle_pins.py
+ * (closed forms, a brute-force Lloyd written separately, library attention
+ * routines, hand-worked toys).  The paper prints no numeric worked example, so
+ * there is no value-level pin against the paper itself.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+static inline float bf16_to_f32(uint16_t b)
+{
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return f;
+}
+
+/*
+ * KMeans(X[:, ch0:ch0+D], C) with `iters` Lloyd iterations.
+ *   X           bf16 bit patterns, row i starts at X + i*row_stride
+ *   U           out, C x D centroids (fp32)
+ *   assign      out, N labels in [0, C): the labels of the last assignment step
+ *   counts      out, C member counts of those labels
+ *   sse         out or NULL, `iters` values: sum of squared distances seen by each
+ *               assignment step
+ *   min_gap     out or NULL, `iters` values: the smallest (d2 - d1) / d2 over all
+ *               rows, d1 <= d2 the two smallest squared distances of the row
+ *               (how close the closest call of that step was)
+ * Returns 0, or -1 on bad arguments.
+ */
+int scope_oracle_kmeans(const uint16_t *X, int64_t N, int64_t row_stride, int ch0, int D, int C,
+                        int iters, float *U, int32_t *assign, int32_t *counts, double *sse,
+                        double *min_gap)
+{
+    if (N <= 0 || D <= 0 || C <= 0 || C > N || iters < 1)
+        return -1;
+    double *sum = (double *)malloc(sizeof(double) * (size_t)C * (size_t)D);
+    if (!sum)
+        return -1;
+
+    /* initial centroid r is token floor(r*N/C) */
+    for (int r = 0; r < C; ++r) {
+        int64_t i = ((int64_t)r * N) / C;
+        for (int ch = 0; ch < D; ++ch)
+            U[(size_t)r * D + ch] = bf16_to_f32(X[i * row_stride + ch0 + ch]);
+    }
+
+    for (int it = 0; it < iters; ++it) {
+        double total = 0.0, gap = 1.0;
+        /* assignment step, Eq. 3 */
+        for (int64_t i = 0; i < N; ++i) {
+            const uint16_t *x = X + i * row_stride + ch0;
+            double best = INFINITY, second = INFINITY;
+            int arg = 0;
+            for (int r = 0; r < C; ++r) {
+                double dist = 0.0;
+                for (int ch = 0; ch < D; ++ch) {
+                    double diff = (double)bf16_to_f32(x[ch]) - (double)U[(size_t)r * D + ch];
+                    dist += diff * diff;
+                }
+                if (dist < best) { /* strict: the lowest index keeps a tie */
+                    second = best;
+                    best = dist;
+                    arg = r;
+                } else if (dist < second) {
+                    second = dist;
+                }
+            }
+            assign[i] = arg;
+            total += best;
+            if (C > 1 && second > 0.0) {
+                double g = (second - best) / second;
+                if (g < gap)
+                    gap = g;
+            } else if (C > 1) {
+                gap = 0.0;
+            }
+        }
+        if (sse)
+            sse[it] = total;
+        if (min_gap)
+            min_gap[it] = gap;
+
+        /* update step: mean of the members, Eq. 2; an empty cluster keeps its centroid */
+        memset(sum, 0, sizeof(double) * (size_t)C * (size_t)D);
+        for (int r = 0; r < C; ++r)
+            counts[r] = 0;
+        for (int64_t i = 0; i < N; ++i) {
+            const uint16_t *x = X + i * row_stride + ch0;
+            double *s = sum + (size_t)assign[i] * D;
+            for (int ch = 0; ch < D; ++ch)
+                s[ch] += (double)bf16_to_f32(x[ch]);
+            counts[assign[i]] += 1;
+        }
+        for (int r = 0; r < C; ++r) {
+            if (counts[r] == 0)
+                continue;
+            for (int ch = 0; ch < D; ++ch)
+                U[(size_t)r * D + ch] = (float)(sum[(size_t)r * D + ch] / (double)counts[r]);
+        }
+    }
+    free(sum);
+    return 0;
+}
+
+/*
+ * Score table of Eq. 5: P[c, r] = < Qbar[c, ch0:ch0+D], U[r, :] >.
+ * Qbar is Cq x d (row stride d), U is C x D, P is Cq x C.  Returns the number of
+ * multiply-accumulates performed (the table cost of the complexity analysis).
+ */
+int64_t scope_oracle_lut(const float *Qbar, int d, int ch0, int D, const float *U, int Cq, int C,
+                         float *P)
+{
+    int64_t macs = 0;
+    for (int c = 0; c < Cq; ++c)
+        for (int r = 0; r < C; ++r) {
+            double acc = 0.0;
+            for (int ch = 0; ch < D; ++ch) {
+                acc += (double)Qbar[(size_t)c * d + ch0 + ch] * (double)U[(size_t)r * D + ch];
+                ++macs;
+            }
+            P[(size_t)c * C + r] = (float)acc;
+        }
+    return macs;
+}
+
+/*
+ * Indexed sum of Eq. 6 for one query cluster, without the 1/sqrt(d) factor:
+ * raw[j] = (PT[zT[j]] + PH[zH[j]]) + PW[zW[j]], evaluated in fp32 in this order.
+ * PT, PH, PW are the rows of the three tables that belong to the query cluster.
+ * Returns the number of table reads (3 per key; there are 2 additions per key).
+ */
+int64_t scope_oracle_scores_row(const float *PT, const float *PH, const float *PW,
+                                const int32_t *zT, const int32_t *zH, const int32_t *zW, int64_t N,
+                                float *raw)
+{
+    for (int64_t j = 0; j < N; ++j) {
+        float a = PT[zT[j]] + PH[zH[j]];
+        raw[j] = a + PW[zW[j]];
+    }
+    return 3 * N;
+}
+
+typedef struct {
+    float v;
+    int32_t j;
+} ranked_t;
+
+static int rank_cmp(const void *pa, const void *pb)
+{
+    const ranked_t *a = (const ranked_t *)pa, *b = (const ranked_t *)pb;
+    if (a->v > b->v)
+        return -1;
+    if (a->v < b->v)
+        return 1;
+    return (a->j > b->j) - (a->j < b->j); /* equal logits: lower key index first */
+}
+
+/*
+ * Ranking pi_c and Top-p count t_c of Eq. 7 for one row of proxy logits.
+ *   raw     N values of scope_oracle_scores_row; the logit is raw[j]*scale (fp32)
+ *   order   out, N key indices by decreasing logit (ties by increasing index)
+ *   t_c     out, the smallest t whose cumulative softmax mass reaches rho
+ *           (N if rho >= 1 or if rounding lets no prefix reach it)
+ *   margin  out or NULL, min(|cum_t - rho Z|, |cum_{t-1} - rho Z|) / Z: how close
+ *           the crossing was
+ */
+int scope_oracle_topp_row(const float *raw, int64_t N, float scale, double rho, int32_t *order,
+                          int32_t *t_c, double *margin)
+{
+    ranked_t *rk = (ranked_t *)malloc(sizeof(ranked_t) * (size_t)N);
+    if (!rk)
+        return -1;
+    for (int64_t j = 0; j < N; ++j) {
+        rk[j].v = raw[j];
+        rk[j].j = (int32_t)j;
+    }
+    qsort(rk, (size_t)N, sizeof(ranked_t), rank_cmp);
+    for (int64_t j = 0; j < N; ++j)
+        order[j] = rk[j].j;
+
+    float mx = rk[0].v * scale; /* row maximum of the logits */
+    double Z = 0.0;
+    for (int64_t j = 0; j < N; ++j) {
+        float s = raw[j] * scale;
+        Z += exp((double)s - (double)mx);
+    }
+    int64_t t = N;
+    double cum = 0.0, m = INFINITY;
+    if (rho < 1.0) {
+        double target = rho * Z;
+        for (int64_t l = 0; l < N; ++l) {
+            float s = rk[l].v * scale;
+            double prev = cum;
+            cum += exp((double)s - (double)mx);
+            if (cum >= target) {
+                t = l + 1;
+                m = fmin(fabs(cum - target), fabs(prev - target)) / Z;
+                break;
+            }
+        }
+    }
+    *t_c = (int32_t)t;
+    if (margin)
+        *margin = m;
+    free(rk);
+    return 0;
+}
+
+/*
+ * Eq. 8 (b_c = max(t_c, k_fix)), Eq. 9 (k_head = ceil(sum n_c b_c / sum n_c), exact
+ * integer arithmetic) and the counts r_c = max(b_c, k_head) of Eq. 10, clamped to N.
+ */
+void scope_oracle_khead(const int32_t *n_c, const int32_t *t_c, int Cq, int64_t N, int32_t k_fix,
+                        int32_t *b_c, int32_t *k_head, int32_t *r_c)
+{
+    int64_t num = 0, den = 0;
+    for (int c = 0; c < Cq; ++c) {
+        b_c[c] = t_c[c] > k_fix ? t_c[c] : k_fix;
+        num += (int64_t)n_c[c] * (int64_t)b_c[c];
+        den += n_c[c];
+    }
+    int64_t k = (num + den - 1) / den;
+    *k_head = (int32_t)k;
+    for (int c = 0; c < Cq; ++c) {
+        int64_t r = b_c[c] > k ? b_c[c] : k;
+        r_c[c] = (int32_t)(r > N ? N : r);
+    }
+}
+
+static int i32_cmp(const void *a, const void *b)
+{
+    int32_t x = *(const int32_t *)a, y = *(const int32_t *)b;
+    return (x > y) - (x < y);
+}
+
+/* S_c of Eq. 10: the first r_c entries of the ranking, stored by ascending key index. */
+void scope_oracle_key_set(const int32_t *order, int32_t r_c, int32_t *S)
+{
+    memcpy(S, order, sizeof(int32_t) * (size_t)r_c);
+    qsort(S, (size_t)r_c, sizeof(int32_t), i32_cmp);
+}
+
+/*
+ * One row of Eq. 11: softmax(q K[S]^T * scale) V[S] for query row q.
+ * q points at the d bf16 values of the query; K, V at token 0 (row stride in
+ * elements); S holds `len` key indices.  out receives d fp32 values.
+ */
+int scope_oracle_attn_row(const uint16_t *q, const uint16_t *K, const uint16_t *V,
+                          int64_t row_stride, int d, const int32_t *S, int64_t len, float scale,
+                          float *out)
+{
+    double *logit = (double *)malloc(sizeof(double) * (size_t)(len > 0 ? len : 1));
+    double *acc = (double *)calloc((size_t)d, sizeof(double));
+    if (!logit || !acc) {
+        free(logit);
+        free(acc);
+        return -1;
+    }
+    double mx = -INFINITY;
+    for (int64_t l = 0; l < len; ++l) {
+        const uint16_t *k = K + (int64_t)S[l] * row_stride;
+        double dot = 0.0;
+        for (int ch = 0; ch < d; ++ch)
+            dot += (double)bf16_to_f32(q[ch]) * (double)bf16_to_f32(k[ch]);
+        logit[l] = dot * (double)scale;
+        if (logit[l] > mx)
+            mx = logit[l];
+    }
+    double Z = 0.0;
+    for (int64_t l = 0; l < len; ++l) {
+        double w = exp(logit[l] - mx);
+        const uint16_t *v = V + (int64_t)S[l] * row_stride;
+        Z += w;
+        for (int ch = 0; ch < d; ++ch)
+            acc[ch] += w * (double)bf16_to_f32(v[ch]);
+    }
+    for (int ch = 0; ch < d; ++ch)
+        out[ch] = len > 0 ? (float)(acc[ch] / Z) : 0.0f;
+    free(logit);
+    free(acc);
+    return 0;
+}
+
+/* One row of Eq. 1: softmax(q K^T * scale) V over all N keys. */
+int scope_oracle_dense_row(const uint16_t *q, const uint16_t *K, const uint16_t *V,
+                           int64_t row_stride, int d, int64_t N, float scale, float *out)
+{
+    double *logit = (double *)malloc(sizeof(double) * (size_t)N);
+    double *acc = (double *)calloc((size_t)d, sizeof(double));
+    if (!logit || !acc) {
+        free(logit);
+        free(acc);
+        return -1;
+    }
+    double mx = -INFINITY;
+    for (int64_t j = 0; j < N; ++j) {
+        double dot = 0.0;
+        for (int ch = 0; ch < d; ++ch)
+            dot += (double)bf16_to_f32(q[ch]) * (double)bf16_to_f32(K[j * row_stride + ch]);
+        logit[j] = dot * (double)scale;
+        if (logit[j] > mx)
+            mx = logit[j];
+    }
+    double Z = 0.0;
+    for (int64_t j = 0; j < N; ++j) {
+        double w = exp(logit[j] - mx);
+        Z += w;
+        for (int ch = 0; ch < d; ++ch)
+            acc[ch] += w * (double)bf16_to_f32(V[j * row_stride + ch]);
+    }
+    for (int ch = 0; ch < d; ++ch)
+        out[ch] = (float)(acc[ch] / Z);
+    free(logit);
+    free(acc);
+    return 0;
+}

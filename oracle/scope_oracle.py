@@ -1,0 +1,236 @@
+"""Python face of the C oracle (oracle/scope_oracle.c).  TEST INFRASTRUCTURE ONLY.
+
+Chains the C steps in the order of Algorithm 1 (one attention head), Algorithm 2
+(key subspace clustering and score tables) and Algorithm 3 (online per-head
+Top-k selection).  Inputs are uint16 arrays of bf16 bit patterns, [N, d] per
+head.  Nothing here may be imported by the CUDA package.
+
+Parity pins: see tests/test_oracle_pins.py.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import dataclasses
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+from . import build_oracle
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build_oracle.build())
+        p = C.c_void_p
+        L.scope_oracle_kmeans.argtypes = [p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, p, p, p, p, p]
+        L.scope_oracle_kmeans.restype = C.c_int
+        L.scope_oracle_lut.argtypes = [p, C.c_int, C.c_int, C.c_int, p, C.c_int, C.c_int, p]
+        L.scope_oracle_lut.restype = C.c_int64
+        L.scope_oracle_scores_row.argtypes = [p, p, p, p, p, p, C.c_int64, p]
+        L.scope_oracle_scores_row.restype = C.c_int64
+        L.scope_oracle_topp_row.argtypes = [p, C.c_int64, C.c_float, C.c_double, p, p, p]
+        L.scope_oracle_topp_row.restype = C.c_int
+        L.scope_oracle_khead.argtypes = [p, p, C.c_int, C.c_int64, C.c_int32, p, p, p]
+        L.scope_oracle_khead.restype = None
+        L.scope_oracle_key_set.argtypes = [p, C.c_int32, p]
+        L.scope_oracle_key_set.restype = None
+        L.scope_oracle_attn_row.argtypes = [p, p, p, C.c_int64, C.c_int, p, C.c_int64, C.c_float, p]
+        L.scope_oracle_attn_row.restype = C.c_int
+        L.scope_oracle_dense_row.argtypes = [p, p, p, C.c_int64, C.c_int, C.c_int64, C.c_float, p]
+        L.scope_oracle_dense_row.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _u16(a) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint16 and a.ndim == 2, "expected bf16 bit patterns [N, d]"
+    return a
+
+
+def kfix_from_alpha(N: int, alpha_num: int, alpha_den: int) -> int:
+    """k_fix = ceil(alpha N) of Eq. 8 for a rational alpha, in exact integers."""
+    return -((-N * alpha_num) // alpha_den)
+
+
+@dataclasses.dataclass
+class KMeansResult:
+    U: np.ndarray  # [C, D] fp32
+    assign: np.ndarray  # [N] int32
+    counts: np.ndarray  # [C] int32
+    sse: np.ndarray  # [iters] fp64
+    min_gap: np.ndarray  # [iters] fp64
+
+
+def kmeans(X, ch0: int, D: int, Cn: int, iters: int) -> KMeansResult:
+    """KMeans(X[:, ch0:ch0+D], C) of Algorithm 1 line 1 / Algorithm 2 line 3."""
+    X = _u16(X)
+    N, d = X.shape
+    U = np.empty((Cn, D), np.float32)
+    a = np.empty(N, np.int32)
+    cnt = np.empty(Cn, np.int32)
+    sse = np.empty(iters, np.float64)
+    gap = np.empty(iters, np.float64)
+    rc = lib().scope_oracle_kmeans(_ptr(X), N, d, ch0, D, Cn, iters, _ptr(U), _ptr(a), _ptr(cnt), _ptr(sse), _ptr(gap))
+    if rc != 0:
+        raise ValueError("scope_oracle_kmeans: bad arguments")
+    return KMeansResult(U, a, cnt, sse, gap)
+
+
+def lut(Qbar: np.ndarray, ch0: int, U: np.ndarray):
+    """P_m = Qbar[:, I_m] U^T (Eq. 5).  Returns (P, multiply-accumulate count)."""
+    Qbar = np.ascontiguousarray(Qbar, np.float32)
+    U = np.ascontiguousarray(U, np.float32)
+    Cq, d = Qbar.shape
+    Cn, D = U.shape
+    P = np.empty((Cq, Cn), np.float32)
+    macs = lib().scope_oracle_lut(_ptr(Qbar), d, ch0, D, _ptr(U), Cq, Cn, _ptr(P))
+    return P, int(macs)
+
+
+def scores_row(PT, PH, PW, zT, zH, zW) -> np.ndarray:
+    """Row c of Eq. 6 without the 1/sqrt(d) factor, fp32: (PT[zT] + PH[zH]) + PW[zW]."""
+    N = zT.shape[0]
+    raw = np.empty(N, np.float32)
+    PT, PH, PW = (np.ascontiguousarray(x, np.float32) for x in (PT, PH, PW))
+    zT, zH, zW = (np.ascontiguousarray(x, np.int32) for x in (zT, zH, zW))
+    lib().scope_oracle_scores_row(_ptr(PT), _ptr(PH), _ptr(PW), _ptr(zT), _ptr(zH), _ptr(zW), N, _ptr(raw))
+    return raw
+
+
+def topp_row(raw: np.ndarray, scale: float, rho: float):
+    """(ranking pi_c, Top-p count t_c, crossing margin) of Eq. 7."""
+    raw = np.ascontiguousarray(raw, np.float32)
+    N = raw.shape[0]
+    order = np.empty(N, np.int32)
+    t = C.c_int32(0)
+    m = C.c_double(0.0)
+    rc = lib().scope_oracle_topp_row(_ptr(raw), N, np.float32(scale), float(rho), _ptr(order), C.byref(t), C.byref(m))
+    if rc != 0:
+        raise MemoryError
+    return order, int(t.value), float(m.value)
+
+
+def khead(n_c, t_c, N: int, k_fix: int):
+    """(b_c, k_head, r_c) of Eq. 8, Eq. 9, Eq. 10."""
+    n_c = np.ascontiguousarray(n_c, np.int32)
+    t_c = np.ascontiguousarray(t_c, np.int32)
+    Cq = n_c.shape[0]
+    b = np.empty(Cq, np.int32)
+    r = np.empty(Cq, np.int32)
+    k = C.c_int32(0)
+    lib().scope_oracle_khead(_ptr(n_c), _ptr(t_c), Cq, N, k_fix, _ptr(b), C.byref(k), _ptr(r))
+    return b, int(k.value), r
+
+
+def key_set(order: np.ndarray, r_c: int) -> np.ndarray:
+    """S_c of Eq. 10 as ascending key indices."""
+    S = np.empty(r_c, np.int32)
+    lib().scope_oracle_key_set(_ptr(np.ascontiguousarray(order, np.int32)), r_c, _ptr(S))
+    return S
+
+
+@dataclasses.dataclass
+class HeadPlan:
+    """Everything Algorithm 1 derives for one head before the attention itself."""
+    Qbar: np.ndarray  # [Cq, d] fp32 query centroids (Eq. 2)
+    g: np.ndarray  # [N] int32 query cluster of every token
+    n_c: np.ndarray  # [Cq] int32
+    U: tuple  # three [C_m, d_m] fp32 codebooks
+    z: tuple  # three [N] int32 code vectors (Eq. 3, Eq. 4)
+    P: tuple  # three [Cq, C_m] fp32 tables (Eq. 5)
+    t_c: np.ndarray
+    b_c: np.ndarray
+    k_head: int
+    r_c: np.ndarray
+    S: list  # Cq ascending int32 index arrays (Eq. 10)
+    kmeans_gap: float  # smallest nearest-centroid gap over all clusterings and iterations
+    topp_margin: float  # smallest Top-p crossing margin over the rows
+    q_sse: np.ndarray  # query k-means SSE per iteration
+
+
+def select_head(P, z, n_c, N: int, scale: float, top_p: float, k_fix: int):
+    """Algorithm 3 given tables, codes and cluster sizes: (t_c, b_c, k_head, r_c, S, margin)."""
+    Cq = P[0].shape[0]
+    orders, t = [], np.empty(Cq, np.int32)
+    margin = np.inf
+    for c in range(Cq):
+        raw = scores_row(P[0][c], P[1][c], P[2][c], z[0], z[1], z[2])
+        order, t[c], m = topp_row(raw, scale, top_p)
+        orders.append(order)
+        margin = min(margin, m)
+    b, k, r = khead(n_c, t, N, k_fix)
+    S = [key_set(orders[c], int(r[c])) for c in range(Cq)]
+    return t, b, k, r, S, margin
+
+
+def plan_head(Q, K, p) -> HeadPlan:
+    """Algorithm 1 lines 1-9 for one head.  ``p`` has d_t/d_h/d_w via ``split``,
+    Cq, Ct, Ch, Cw, iters, top_p, k_fix, scale."""
+    Q, K = _u16(Q), _u16(K)
+    N, d = Q.shape
+    d_t, d_h, d_w = p.split
+    assert d_t + d_h + d_w == d
+    kq = kmeans(Q, 0, d, p.Cq, p.iters)
+    ranges = ((0, d_t, p.Ct), (d_t, d_h, p.Ch), (d_t + d_h, d_w, p.Cw))
+    ks = [kmeans(K, ch0, D, Cn, p.iters) for ch0, D, Cn in ranges]
+    P = tuple(lut(kq.U, ch0, km.U)[0] for (ch0, _, _), km in zip(ranges, ks))
+    z = tuple(km.assign for km in ks)
+    t, b, k, r, S, margin = select_head(P, z, kq.counts, N, p.scale, p.top_p, p.k_fix)
+    gap = min(float(kq.min_gap.min()), *(float(km.min_gap.min()) for km in ks))
+    return HeadPlan(kq.U, kq.assign, kq.counts, tuple(km.U for km in ks), z, P, t, b, k, r, S, gap, margin, kq.sse)
+
+
+def attention_rows(Q, K, V, g, S, scale: float, rows) -> np.ndarray:
+    """Rows of Eq. 11: query i attends to the key set of its cluster g[i]."""
+    Q, K, V = _u16(Q), _u16(K), _u16(V)
+    N, d = Q.shape
+    rows = np.asarray(rows, np.int64)
+    out = np.empty((rows.shape[0], d), np.float32)
+    o = np.empty(d, np.float32)
+    for n, i in enumerate(rows):
+        Sc = np.ascontiguousarray(S[int(g[i])], np.int32)
+        rc = lib().scope_oracle_attn_row(_ptr(Q[i]), _ptr(K), _ptr(V), d, d, _ptr(Sc), Sc.shape[0], np.float32(scale), _ptr(o))
+        if rc != 0:
+            raise MemoryError
+        out[n] = o
+    return out
+
+
+def dense_rows(Q, K, V, scale: float, rows) -> np.ndarray:
+    """Rows of Eq. 1."""
+    Q, K, V = _u16(Q), _u16(K), _u16(V)
+    N, d = Q.shape
+    rows = np.asarray(rows, np.int64)
+    out = np.empty((rows.shape[0], d), np.float32)
+    o = np.empty(d, np.float32)
+    for n, i in enumerate(rows):
+        rc = lib().scope_oracle_dense_row(_ptr(Q[i]), _ptr(K), _ptr(V), d, d, N, np.float32(scale), _ptr(o))
+        if rc != 0:
+            raise MemoryError
+        out[n] = o
+    return out
+
+
+def forward_head(Q, K, V, p):
+    """Algorithm 1 for one head: (O [N, d] fp32, HeadPlan)."""
+    plan = plan_head(Q, K, p)
+    O = attention_rows(Q, K, V, plan.g, plan.S, p.scale, np.arange(Q.shape[0]))
+    return O, plan
+
+
+def plan_layer(Q, K, p, threads: int = 1) -> list:
+    """plan_head for every (batch, head) of [B, H, N, d] inputs; heads are independent."""
+    B, H = Q.shape[:2]
+    jobs = [(b, h) for b in range(B) for h in range(H)]
+    if threads <= 1:
+        return [plan_head(Q[b, h], K[b, h], p) for b, h in jobs]
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        return list(ex.map(lambda bh: plan_head(Q[bh[0], bh[1]], K[bh[0], bh[1]], p), jobs))

@@ -1,0 +1,175 @@
+"""Seeded synthetic Q/K/V shaped like the attention layers of video DiTs.
+
+This module only *draws inputs*; it contains none of the method's arithmetic and
+is shared by the CPU oracle's tests and by the CUDA path so that both see the
+same bits.
+
+Recipe (per tensor X in {Q, K}, per (batch, head)):
+  * token n <-> grid position (t, h, w), n = (t*Hg + h)*Wg + w (t-major);
+  * per channel: mean mu ~ N(0, 4); for every axis a in (t, h, w) two
+    coefficients A_a, B_a ~ N(0, 1); noise eps[n, ch] ~ N(0, 1);
+    x = mu + sum_a (A_a sin(2 pi p_a / P_a) + B_a cos(2 pi p_a / P_a)) + eps,
+    rounded to bf16;
+  * 3D RoPE (theta = 1e4) applied per channel subspace [T | H | W] on
+    interleaved pairs (2i, 2i+1) with frequency theta^(-2i/d_m) and the
+    position of that subspace's axis, evaluated in fp32 and rounded to bf16;
+  * V ~ N(0, 1), rounded to bf16.
+All random numbers come from numpy's counter-based Philox generator keyed by
+(seed, tensor, batch, head) and are drawn in a fixed order, so any head can be
+generated on its own.
+
+Tensors are returned as uint16 arrays holding bf16 bit patterns, shape
+[B, H, N, d].
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROPE_THETA = 1.0e4
+
+
+@dataclasses.dataclass(frozen=True)
+class ScopeConfig:
+    name: str
+    B: int
+    H: int
+    grid: tuple  # (Tg, Hg, Wg)
+    split: tuple  # (d_t, d_h, d_w)
+    Cq: int
+    Ct: int
+    Ch: int
+    Cw: int
+    iters: int
+    top_p: float
+    k_fix: int
+
+    @property
+    def N(self) -> int:
+        return self.grid[0] * self.grid[1] * self.grid[2]
+
+    @property
+    def d(self) -> int:
+        return sum(self.split)
+
+    @property
+    def scale(self) -> float:
+        return 1.0 / math.sqrt(self.d)
+
+    def replace(self, **kw) -> "ScopeConfig":
+        return dataclasses.replace(self, **kw)
+
+
+CONFIGS = {
+    "tiny": ScopeConfig("tiny", 1, 2, (4, 8, 8), (16, 56, 56), 8, 4, 8, 8, 5, 0.9, 32),
+    "small": ScopeConfig("small", 1, 8, (9, 16, 16), (16, 56, 56), 32, 8, 16, 16, 5, 0.9, 64),
+    "W480": ScopeConfig("W480", 1, 40, (21, 30, 52), (44, 42, 42), 128, 16, 64, 64, 5, 0.9, 256),
+    "W720": ScopeConfig("W720", 1, 40, (21, 45, 80), (44, 42, 42), 128, 16, 64, 64, 5, 0.9, 512),
+    "HY720": ScopeConfig("HY720", 1, 24, (33, 45, 80), (16, 56, 56), 128, 16, 64, 64, 5, 0.9, 512),
+}
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round-to-nearest-even fp32 -> bf16, returned as uint16 bit patterns."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))
+    return (r >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def _rng(seed: int, tensor: int, b: int, h: int) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=[int(seed), (tensor << 40) | (b << 20) | h]))
+
+
+def grid_positions(grid) -> tuple:
+    Tg, Hg, Wg = grid
+    n = np.arange(Tg * Hg * Wg)
+    return (n // (Hg * Wg), (n // Wg) % Hg, n % Wg)
+
+
+def _rope_tables(grid, split):
+    """cos/sin [N, d/2] (fp32) for interleaved pairs of the three subspaces."""
+    pos = grid_positions(grid)
+    cs, sn = [], []
+    for dm, p in zip(split, pos):
+        assert dm % 2 == 0
+        i = np.arange(dm // 2, dtype=np.float64)
+        w = ROPE_THETA ** (-2.0 * i / dm)
+        ang = p.astype(np.float64)[:, None] * w[None, :]
+        cs.append(np.cos(ang).astype(np.float32))
+        sn.append(np.sin(ang).astype(np.float32))
+    return np.concatenate(cs, 1), np.concatenate(sn, 1)
+
+
+def _harmonics(grid):
+    """sin/cos of 2 pi p_a / P_a per axis, fp32 [3, N]."""
+    pos = grid_positions(grid)
+    s = np.stack([np.sin(2.0 * np.pi * p / P) for p, P in zip(pos, grid)]).astype(np.float32)
+    c = np.stack([np.cos(2.0 * np.pi * p / P) for p, P in zip(pos, grid)]).astype(np.float32)
+    return s, c
+
+
+def _qk_head(cfg: ScopeConfig, seed: int, tensor: int, b: int, h: int, harm, rope) -> np.ndarray:
+    N, d = cfg.N, cfg.d
+    g = _rng(seed, tensor, b, h)
+    mu = (2.0 * g.standard_normal(d)).astype(np.float32)
+    coef = g.standard_normal((3, 2, d)).astype(np.float32)  # [axis, (A, B), ch]
+    x = g.standard_normal((N, d), dtype=np.float32)
+    x += mu[None, :]
+    hs, hc = harm
+    for a in range(3):
+        x += hs[a][:, None] * coef[a, 0][None, :]
+        x += hc[a][:, None] * coef[a, 1][None, :]
+    x = bf16_bits_to_f32(f32_to_bf16_bits(x))
+    cs, sn = rope
+    xe, xo = x[:, 0::2], x[:, 1::2]
+    out = np.empty_like(x)
+    out[:, 0::2] = xe * cs - xo * sn
+    out[:, 1::2] = xe * sn + xo * cs
+    return f32_to_bf16_bits(out)
+
+
+def _v_head(cfg: ScopeConfig, seed: int, b: int, h: int) -> np.ndarray:
+    g = _rng(seed, 2, b, h)
+    return f32_to_bf16_bits(g.standard_normal((cfg.N, cfg.d), dtype=np.float32))
+
+
+def make_head(cfg: ScopeConfig, seed: int, b: int, h: int, _tables=None):
+    """(Q, K, V) bf16 bit patterns [N, d] of one (batch, head)."""
+    harm, rope = _tables if _tables is not None else (_harmonics(cfg.grid), _rope_tables(cfg.grid, cfg.split))
+    return (_qk_head(cfg, seed, 0, b, h, harm, rope), _qk_head(cfg, seed, 1, b, h, harm, rope),
+            _v_head(cfg, seed, b, h))
+
+
+def make_qkv(cfg: ScopeConfig, seed: int = 0, threads: int = 8, batch_offset: int = 0, out=None):
+    """(Q, K, V) uint16 arrays [B, H, N, d]; heads are generated independently.
+
+    ``batch_offset`` shifts the batch index used for the random streams, so that
+    several processes can each draw their own slice of one larger batch.
+    ``out`` may hold three preallocated uint16 arrays (e.g. views of pinned
+    host memory).
+    """
+    B, H, N, d = cfg.B, cfg.H, cfg.N, cfg.d
+    if out is None:
+        out = tuple(np.empty((B, H, N, d), dtype=np.uint16) for _ in range(3))
+    Q, K, V = out
+    tables = (_harmonics(cfg.grid), _rope_tables(cfg.grid, cfg.split))
+
+    def work(bh):
+        b, h = divmod(bh, H)
+        q, k, v = make_head(cfg, seed, b + batch_offset, h, tables)
+        Q[b, h], K[b, h], V[b, h] = q, k, v
+
+    if threads <= 1:
+        for bh in range(B * H):
+            work(bh)
+    else:
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(work, range(B * H)))
+    return Q, K, V

@@ -1,0 +1,386 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests calls the CUDA path.  Each one is chosen so that a plausible
+mistake in the oracle (dropped term, wrong sign, transposed operand, wrong
+weighting, wrong tie rule) makes it fail.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import scope_oracle as orc
+from paper_2608_12780_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _golden(name):
+    out = {}
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if not line:
+                continue
+            tok = line.split()
+            try:
+                float(tok[0])
+                rows.append([float(t) for t in tok])
+            except ValueError:
+                out[tok[0]] = [float(t) for t in tok[1:]]
+    out["rows"] = rows
+    return out
+
+
+def _bits(x):
+    return inputs.f32_to_bf16_bits(np.asarray(x, np.float32))
+
+
+def _f32(b):
+    return inputs.bf16_bits_to_f32(b)
+
+
+def _head(name="tiny", seed=0, h=0):
+    cfg = inputs.CONFIGS[name]
+    Q, K, V = inputs.make_head(cfg, seed, 0, h)
+    return cfg, Q, K, V
+
+
+# ----------------------------------------------------------------------------- k-means
+
+
+def test_kmeans_1d_toy_matches_hand_worked():
+    g = _golden("kmeans_1d_toy.txt")
+    X = _bits(np.array(g["x"], np.float32)[:, None])
+    for iters in (1, 2, 5):
+        r = orc.kmeans(X, 0, 1, 2, iters)
+        assert r.assign.tolist() == [int(v) for v in g["assign"]]
+        assert r.U[:, 0].tolist() == g["centroids"]
+        assert r.counts.tolist() == [3, 3]
+
+
+def _lloyd_bruteforce(X, C, iters):
+    """Separately written Lloyd iteration in numpy fp64 (vectorised, library argmin)."""
+    N = X.shape[0]
+    U = X[(np.arange(C) * N) // C].astype(np.float32)
+    hist = []
+    for _ in range(iters):
+        d2 = ((X[:, None, :].astype(np.float64) - U[None, :, :].astype(np.float64)) ** 2).sum(-1)
+        a = d2.argmin(1)  # numpy returns the first minimum
+        hist.append((U.copy(), a.copy(), d2.min(1).sum()))
+        for r in range(C):
+            if (a == r).any():
+                U[r] = X[a == r].astype(np.float64).mean(0).astype(np.float32)
+    return U, a, hist
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_kmeans_matches_bruteforce_lloyd(seed):
+    rng = np.random.default_rng(seed)
+    N, d, C, iters = 97, 6, 5, 7
+    Xb = _bits(rng.normal(size=(N, d)) + 3.0 * rng.integers(0, 3, size=(N, 1)))
+    X = _f32(Xb)
+    r = orc.kmeans(Xb, 0, d, C, iters)
+    U, a, hist = _lloyd_bruteforce(X, C, iters)
+    assert np.array_equal(r.assign, a)
+    assert np.allclose(r.U, U, rtol=0, atol=1e-6)
+    assert np.array_equal(r.counts, np.bincount(a, minlength=C))
+    # the objective seen by successive assignment steps never increases
+    assert np.all(np.diff(r.sse) <= 1e-9 * r.sse[:-1])
+    assert np.allclose(r.sse, [h[2] for h in hist], rtol=1e-12)
+    # every returned label is an argmin w.r.t. the centroids its assignment step saw
+    U_prev = hist[-1][0].astype(np.float64)
+    d2 = ((X[:, None, :] - U_prev[None]) ** 2).sum(-1)
+    assert np.array_equal(d2.argmin(1), r.assign)
+    # returned centroids are the means of exactly the returned members (Eq. 2)
+    for c in range(C):
+        if r.counts[c]:
+            assert np.allclose(r.U[c], X[r.assign == c].mean(0), atol=1e-6)
+
+
+def test_kmeans_subspace_reads_only_its_channels():
+    cfg, Q, K, V = _head("tiny")
+    ch0, D = cfg.split[0], cfg.split[1]
+    a = orc.kmeans(K, ch0, D, 8, 3)
+    Kc = np.ascontiguousarray(K[:, ch0:ch0 + D])
+    b = orc.kmeans(Kc, 0, D, 8, 3)
+    assert np.array_equal(a.assign, b.assign) and np.array_equal(a.U, b.U)
+    K2 = K.copy()
+    K2[:, :ch0] = 0
+    K2[:, ch0 + D:] = 0x3F80
+    c = orc.kmeans(K2, ch0, D, 8, 3)
+    assert np.array_equal(a.assign, c.assign)
+
+
+def test_kmeans_ties_and_empty_clusters():
+    # two identical initial centroids: the lower index takes every tied token, the
+    # other cluster is empty and keeps its centroid
+    x = np.array([[1.0], [5.0], [1.0], [5.0]], np.float32)  # init tokens 0 and 2 -> 1, 1
+    r = orc.kmeans(_bits(x), 0, 1, 2, 1)
+    assert r.assign.tolist() == [0, 0, 0, 0]
+    assert r.counts.tolist() == [4, 0]
+    assert r.U[:, 0].tolist() == [3.0, 1.0]
+    assert r.min_gap.min() == 0.0
+    # the kept centroid is live again in the next iteration
+    r = orc.kmeans(_bits(x), 0, 1, 2, 2)
+    assert r.assign.tolist() == [1, 0, 1, 0] and r.U[:, 0].tolist() == [5.0, 1.0]
+
+
+def test_kmeans_rejects_bad_arguments():
+    X = _bits(np.zeros((4, 2), np.float32))
+    with pytest.raises(ValueError):
+        orc.kmeans(X, 0, 2, 5, 1)  # more clusters than tokens
+    with pytest.raises(ValueError):
+        orc.kmeans(X, 0, 2, 2, 0)
+
+
+# ----------------------------------------------------------------------------- tables and proxy logits
+
+
+def test_lut_is_the_sliced_matrix_product_and_counts_macs():
+    rng = np.random.default_rng(3)
+    Cq, d, ch0, D, C = 5, 12, 4, 6, 7
+    Qbar = rng.normal(size=(Cq, d)).astype(np.float32)
+    U = rng.normal(size=(C, D)).astype(np.float32)
+    P, macs = orc.lut(Qbar, ch0, U)
+    ref = Qbar[:, ch0:ch0 + D].astype(np.float64) @ U.astype(np.float64).T
+    assert P.shape == (Cq, C)
+    assert np.allclose(P, ref, rtol=0, atol=1e-6)
+    assert macs == Cq * C * D
+
+
+def test_table_cost_matches_complexity_analysis():
+    # T_table = Cq * sum_m C_m d_m ; T_direct = Cq * N * d ; equal codebooks: ratio N / C
+    cfg, Q, K, V = _head("tiny")
+    pl = orc.plan_head(Q, K, cfg)
+    macs = 0
+    ch0 = 0
+    for U, dm in zip(pl.U, cfg.split):
+        macs += orc.lut(pl.Qbar, ch0, U)[1]
+        ch0 += dm
+    assert macs == cfg.Cq * (cfg.Ct * cfg.split[0] + cfg.Ch * cfg.split[1] + cfg.Cw * cfg.split[2])
+    Cn = 8
+    eq = Cn * cfg.Cq * cfg.d
+    assert (cfg.Cq * cfg.N * cfg.d) / eq == cfg.N / Cn
+    # three reads per (cluster, key) pair
+    reads = orc.lib().scope_oracle_scores_row  # exercised below; here the count
+    raw = np.empty(cfg.N, np.float32)
+    n = reads(*(orc._ptr(np.ascontiguousarray(x)) for x in (pl.P[0][0], pl.P[1][0], pl.P[2][0], pl.z[0], pl.z[1], pl.z[2])),
+              cfg.N, orc._ptr(raw))
+    assert n == 3 * cfg.N
+
+
+def test_lookup_sum_equals_inner_product_with_product_code_representative():
+    # s~_{c,j} = <qbar_c, concat_m u^m_{z_j^m}> / sqrt(d): lookup-and-sum adds no approximation
+    cfg, Q, K, V = _head("small")
+    pl = orc.plan_head(Q, K, cfg)
+    khat = np.concatenate([pl.U[m][pl.z[m]] for m in range(3)], axis=1).astype(np.float64)  # [N, d]
+    ref = pl.Qbar.astype(np.float64) @ khat.T  # [Cq, N]
+    for c in (0, 7, cfg.Cq - 1):
+        raw = orc.scores_row(pl.P[0][c], pl.P[1][c], pl.P[2][c], *pl.z)
+        assert np.allclose(raw, ref[c], rtol=0, atol=2e-4)
+    # and each code is the nearest centroid of its own slice w.r.t. the centroids of the last assignment step:
+    # checked in test_kmeans_matches_bruteforce_lloyd; here the codes are at least in range
+    for m, Cm in enumerate((cfg.Ct, cfg.Ch, cfg.Cw)):
+        assert pl.z[m].min() >= 0 and pl.z[m].max() < Cm
+
+
+def test_one_token_per_cluster_gives_exact_qk():
+    # C_q = N and C_m = N: every token is its own centroid, so the proxy logit is q_c . k_j / sqrt(d)
+    cfg = inputs.CONFIGS["tiny"].replace(grid=(2, 4, 4), Cq=32, Ct=32, Ch=32, Cw=32, k_fix=4)
+    Q, K, V = inputs.make_head(cfg, 5, 0, 0)
+    N = cfg.N
+    kq = orc.kmeans(Q, 0, cfg.d, N, cfg.iters)
+    assert np.array_equal(kq.assign, np.arange(N)) and np.array_equal(kq.U, _f32(Q))
+    P, z, ch0 = [], [], 0
+    for dm in cfg.split:
+        km = orc.kmeans(K, ch0, dm, N, cfg.iters)
+        # duplicates of a slice would merge clusters; the centroid of a token's cluster is still the token's slice
+        assert np.array_equal(km.U[km.assign], _f32(K)[:, ch0:ch0 + dm])
+        P.append(orc.lut(kq.U, ch0, km.U)[0])
+        z.append(km.assign)
+        ch0 += dm
+    exact = _f32(Q).astype(np.float64) @ _f32(K).astype(np.float64).T
+    for c in range(N):
+        raw = orc.scores_row(P[0][c], P[1][c], P[2][c], *z)
+        assert np.allclose(raw, exact[c], rtol=1e-5, atol=1e-5 * np.abs(exact[c]).max())
+
+
+def test_scores_row_addition_order_is_fp32_left_to_right():
+    PT = np.array([1.0e8], np.float32)
+    PH = np.array([-1.0e8], np.float32)
+    PW = np.array([1.0], np.float32)
+    z0 = np.zeros(1, np.int32)
+    assert orc.scores_row(PT, PH, PW, z0, z0, z0)[0] == 1.0  # (1e8 - 1e8) + 1, not 1e8 + (-1e8 + 1)
+
+
+# ----------------------------------------------------------------------------- Top-p, per-head k, key sets
+
+
+def test_topp_toy_matches_hand_worked():
+    g = _golden("topp_toy.txt")
+    mass = {2: 0.5, 0: 0.2, 3: 0.2, 1: 0.1}  # key index -> softmax mass
+    raw = np.array([math.log(mass[j]) for j in range(4)], np.float32)
+    for rho, t in g["rows"]:
+        order, tc, margin = orc.topp_row(raw, 1.0, rho)
+        assert order.tolist() == [2, 0, 3, 1]  # equal masses: lower key index first
+        assert tc == int(t)
+        assert margin > 0.04
+    # a common scale factor changes the distribution, not the ranking
+    order, tc, _ = orc.topp_row(raw, 0.5, 0.45)
+    assert order.tolist() == [2, 0, 3, 1] and tc == 2  # masses ~ sqrt: .354 .224 .224 .158 of 1.158 -> .306 .499
+    # rho = 1 keeps everything
+    assert orc.topp_row(raw, 1.0, 1.0)[1] == 4
+
+
+def test_topp_all_equal_logits():
+    N, rho = 37, 0.9  # rho*N = 33.3 -> 34 keys
+    order, tc, _ = orc.topp_row(np.full(N, 0.25, np.float32), 0.3, rho)
+    assert order.tolist() == list(range(N))
+    assert tc == math.ceil(rho * N)
+    assert orc.key_set(order, tc).tolist() == list(range(tc))
+
+
+def test_topp_against_sorted_cumsum():
+    rng = np.random.default_rng(11)
+    raw = (rng.normal(size=500) * 30).astype(np.float32)
+    scale = np.float32(1 / math.sqrt(128))
+    for rho in (0.05, 0.5, 0.9, 0.999):
+        order, tc, _ = orc.topp_row(raw, scale, rho)
+        s = (raw * scale).astype(np.float64)
+        a = np.exp(s - s.max())
+        a /= a.sum()
+        ref_order = np.argsort(-raw, kind="stable")
+        assert np.array_equal(order, ref_order)
+        assert tc == int(np.searchsorted(np.cumsum(a[ref_order]), rho) + 1)
+
+
+def test_khead_toy_matches_hand_worked():
+    g = _golden("khead_toy.txt")
+    n = np.array(g["n"], np.int32)
+    t = np.array(g["t"], np.int32)
+    b, k, r = orc.khead(n, t, int(n.sum()), int(g["k_fix"][0]))
+    assert b.tolist() == g["b"] and k == g["k_head"][0] and r.tolist() == g["r"]
+    # the unweighted mean of b would round up to 4: the weighting matters
+    assert math.ceil(b.mean()) == 4
+
+
+def test_khead_is_the_per_query_mean():
+    rng = np.random.default_rng(4)
+    for _ in range(20):
+        Cq, N = 9, 400
+        g = rng.integers(0, Cq, size=N)
+        n = np.bincount(g, minlength=Cq).astype(np.int32)
+        t = rng.integers(1, N + 1, size=Cq).astype(np.int32)
+        k_fix = int(rng.integers(1, N))
+        b, k, r = orc.khead(n, t, N, k_fix)
+        assert np.array_equal(b, np.maximum(t, k_fix))
+        num = int(b[g].astype(np.int64).sum())
+        assert k == -(-num // N)
+        assert b.min() <= k <= b.max()
+        assert np.array_equal(r, np.minimum(N, np.maximum(b, k)))
+
+
+def test_kfix_from_alpha_is_exact():
+    assert orc.kfix_from_alpha(118800, 1, 10) == 11880  # float32 0.1 * 118800 would round up to 11881
+    assert orc.kfix_from_alpha(75600, 1, 10) == 7560
+    assert orc.kfix_from_alpha(7, 1, 10) == 1
+    assert orc.kfix_from_alpha(10, 1, 1) == 10
+
+
+@pytest.mark.parametrize("name", ["tiny", "small"])
+def test_selection_invariants(name):
+    cfg, Q, K, V = _head(name, seed=1)
+    pl = orc.plan_head(Q, K, cfg)
+    N = cfg.N
+    assert pl.n_c.sum() == N and np.array_equal(pl.n_c, np.bincount(pl.g, minlength=cfg.Cq))
+    assert pl.b_c.min() <= pl.k_head <= pl.b_c.max()
+    scale = np.float32(cfg.scale)
+    for c in range(cfg.Cq):
+        S = pl.S[c]
+        r = int(pl.r_c[c])
+        assert S.shape[0] == r and np.all(np.diff(S) > 0)
+        assert r >= pl.k_head >= cfg.k_fix and r >= pl.b_c[c] >= pl.t_c[c]
+        # clusters at or above the per-head k are left alone, the others are extended to exactly k
+        assert r == (pl.b_c[c] if pl.b_c[c] >= pl.k_head else pl.k_head)
+        raw = orc.scores_row(pl.P[0][c], pl.P[1][c], pl.P[2][c], *pl.z)
+        inside = np.zeros(N, bool)
+        inside[S] = True
+        if r < N:
+            assert raw[inside].min() >= raw[~inside].max()
+            # ties at the boundary go to the lower key index
+            tie = raw == raw[inside].min()
+            if (tie & ~inside).any():
+                assert np.flatnonzero(tie & inside).max() < np.flatnonzero(tie & ~inside).min()
+        a = np.exp((raw * scale).astype(np.float64) - float((raw * scale).max()))
+        a /= a.sum()
+        assert a[inside].sum() >= cfg.top_p - 1e-12
+        # t_c is minimal: dropping the weakest of the first t_c keys falls below rho
+        order = np.argsort(-raw, kind="stable")
+        assert a[order[: pl.t_c[c] - 1]].sum() < cfg.top_p
+
+
+def test_key_sets_are_nested_in_rho_and_floor():
+    cfg, Q, K, V = _head("tiny", seed=2)
+    pl = orc.plan_head(Q, K, cfg)
+    args = (pl.P, pl.z, pl.n_c, cfg.N, cfg.scale)
+    base = orc.select_head(*args, 0.8, 16)
+    for rho, kf in ((0.9, 16), (0.8, 40), (0.95, 64)):
+        big = orc.select_head(*args, rho, kf)
+        for c in range(cfg.Cq):
+            assert set(base[4][c].tolist()) <= set(big[4][c].tolist())
+
+
+def test_rho_to_zero_gives_floor_only():
+    cfg, Q, K, V = _head("tiny", seed=3)
+    pl = orc.plan_head(Q, K, cfg)
+    t, b, k, r, S, _ = orc.select_head(pl.P, pl.z, pl.n_c, cfg.N, cfg.scale, 1e-30, cfg.k_fix)
+    assert np.all(t == 1) and np.all(b == cfg.k_fix) and k == cfg.k_fix and np.all(r == cfg.k_fix)
+
+
+# ----------------------------------------------------------------------------- attention
+
+
+def _sdpa(Q, K, V, scale, mask=None):
+    q, k, v = (torch.from_numpy(_f32(x).astype(np.float64))[None, None] for x in (Q, K, V))
+    o = torch.nn.functional.scaled_dot_product_attention(q, k, v, attn_mask=mask, scale=float(np.float32(scale)))
+    return o[0, 0].numpy()
+
+
+def test_rho_one_equals_dense_attention():
+    cfg, Q, K, V = _head("tiny", seed=4)
+    O, pl = orc.forward_head(Q, K, V, cfg.replace(top_p=1.0))
+    assert all(s.shape[0] == cfg.N for s in pl.S) and np.all(pl.t_c == cfg.N)
+    rows = np.arange(cfg.N)
+    dense = orc.dense_rows(Q, K, V, cfg.scale, rows)
+    assert np.allclose(O, dense, rtol=0, atol=1e-6)
+    assert np.allclose(dense, _sdpa(Q, K, V, cfg.scale), rtol=0, atol=2e-6)
+
+
+def test_sparse_attention_equals_masked_dense_attention():
+    cfg, Q, K, V = _head("tiny", seed=5)
+    O, pl = orc.forward_head(Q, K, V, cfg)
+    mask = torch.zeros(cfg.N, cfg.N, dtype=torch.bool)
+    for i in range(cfg.N):
+        mask[i, torch.from_numpy(pl.S[pl.g[i]].astype(np.int64))] = True
+    ref = _sdpa(Q, K, V, cfg.scale, mask[None, None])
+    assert np.allclose(O, ref, rtol=0, atol=2e-6)
+    # the selection must matter for this pin to bite
+    assert not np.allclose(O, _sdpa(Q, K, V, cfg.scale), atol=1e-3)
+
+
+def test_attention_uses_original_tokens_only():
+    # once S_c is fixed the output row is a softmax-weighted mean of the selected original value rows
+    cfg, Q, K, V = _head("tiny", seed=6)
+    pl = orc.plan_head(Q, K, cfg)
+    rows = np.arange(0, cfg.N, 7)
+    a = orc.attention_rows(Q, K, V, pl.g, pl.S, cfg.scale, rows)
+    q, k, v = (_f32(x).astype(np.float64) for x in (Q, K, V))
+    for n, i in enumerate(rows):
+        S = pl.S[pl.g[i]]
+        l = (k[S] @ q[i]) * float(np.float32(cfg.scale))
+        w = np.exp(l - l.max())
+        assert np.allclose(a[n], (w[:, None] * v[S]).sum(0) / w.sum(), rtol=0, atol=1e-6)
