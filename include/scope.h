@@ -1,0 +1,201 @@
+/*
+ * scope.h — C ABI of the SCOPE sparse-attention layer for NVIDIA B200 (sm_100a).
+ *
+ * SCOPE (Subspace Clustering with Online Per-head Top-k Estimation) replaces the
+ * dense attention of one video-DiT layer by, per attention head (Algorithm 1):
+ *   1. k-means of the post-RoPE queries over all d channels (Eq. 2);
+ *   2. k-means of the post-RoPE keys, independently in the temporal, height and
+ *      width channel ranges; the three labels form each key's code (Eq. 3, Eq. 4);
+ *   3. one score table per range, query centroid slice x key centroid (Eq. 5);
+ *   4. a proxy logit per (query cluster, key): the sum of three table reads (Eq. 6);
+ *   5. per query cluster, the Top-p count of the proxy softmax (Eq. 7), floored by a
+ *      fixed count (Eq. 8); the per-head k as the query-weighted mean of those
+ *      counts (Eq. 9); clusters below it are extended along the same ranking (Eq. 10);
+ *   6. exact attention of every query over the selected original keys/values (Eq. 11).
+ *
+ * General conventions
+ *   - Q, K, V, O are DEVICE pointers owned by the caller: bf16, logical shape
+ *     [B, H, N, d] with d = 128 contiguous, 16-byte aligned, strides in elements
+ *     given in scope_params.  Only O is ever written.
+ *   - The library allocates no device memory.  The caller provides one workspace of
+ *     scope_plan_workspace_bytes() bytes (256-byte aligned) that holds every plan
+ *     array and all scratch; a scope_plan_t is a small host object of views into it
+ *     and stays valid while the workspace does.
+ *   - scope_plan / scope_sparse_attn / scope_forward only enqueue work on `stream`
+ *     and return; they report host-detectable errors.  Conditions found on the
+ *     device (index buffer too small, malformed imported plan) are written to a
+ *     status word inside the workspace and read back by scope_plan_status().
+ *   - Nothing is thread-safe per plan: one plan, one stream at a time.
+ *   - Inputs are assumed finite.  Behaviour on NaN/Inf is unspecified but stays in
+ *     bounds and terminates.
+ *   - Every function returning scope_status returns SCOPE_OK on success.
+ */
+#ifndef SCOPE_H
+#define SCOPE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SCOPE_OK = 0,
+    SCOPE_ERR_INVALID_ARG = 1, /* null pointer, parameter out of range */
+    SCOPE_ERR_UNSUPPORTED = 2, /* valid in the paper, not built (e.g. d != 128) */
+    SCOPE_ERR_ALIGNMENT = 3,   /* pointer or stride breaks the 16-byte rule */
+    SCOPE_ERR_WORKSPACE = 4,   /* workspace smaller than scope_plan_workspace_bytes() */
+    SCOPE_ERR_CAPACITY = 5,    /* index_capacity too small for the selected key sets */
+    SCOPE_ERR_BAD_PLAN = 6,    /* imported plan arrays are inconsistent */
+    SCOPE_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired */
+    SCOPE_ERR_CUDA = 8         /* a CUDA runtime call failed */
+} scope_status;
+
+/* Problem statement of Algorithm 1 ("Require" line) plus layout. */
+typedef struct {
+    int32_t B, H, N, d;       /* batch, heads, tokens per head, head dim (128) */
+    int32_t d_t, d_h, d_w;    /* contiguous channel ranges [T | H | W]; each > 0; sum == d */
+    int32_t Cq, Ct, Ch, Cw;   /* cluster counts: queries, key ranges; 1 <= C <= min(N, 1024) */
+    int32_t kmeans_iters;     /* Lloyd iterations, >= 1, fixed (no early exit) */
+    float top_p;              /* rho of Eq. 7, in (0, 1]; >= 1 keeps every key */
+    int32_t k_fix;            /* floor of Eq. 8 as an absolute count, 1..N */
+    float scale;              /* logit scale of Eq. 1 / Eq. 6; 0 selects 1/sqrt(d) */
+    int64_t stride_b, stride_h, stride_n; /* elements; all 0 selects dense [B,H,N,d] */
+    int64_t index_capacity;   /* entries the key-index buffer can hold, summed over all
+                                 (batch, head, query cluster) */
+} scope_params;
+
+typedef struct scope_plan_s scope_plan_t; /* opaque host object */
+
+/* Arrays of a plan.  Shapes are per plan: BH = B*H.  "int32" arrays are exported
+ * and imported as int32 whatever the internal packing. */
+typedef enum {
+    SCOPE_Q_CENTROIDS = 0,  /* float [BH, Cq, d]      query centroids, Eq. 2 */
+    SCOPE_K_CENTROIDS_T,    /* float [BH, Ct, d_t]    key codebooks, Eq. 3 */
+    SCOPE_K_CENTROIDS_H,    /* float [BH, Ch, d_h] */
+    SCOPE_K_CENTROIDS_W,    /* float [BH, Cw, d_w] */
+    SCOPE_Q_ASSIGN,         /* int32 [BH, N]          g_i */
+    SCOPE_K_CODES_T,        /* int32 [BH, N]          z_j^T, Eq. 4 */
+    SCOPE_K_CODES_H,        /* int32 [BH, N] */
+    SCOPE_K_CODES_W,        /* int32 [BH, N] */
+    SCOPE_CLUSTER_SIZES,    /* int32 [BH, Cq]         n_c */
+    SCOPE_LUT_T,            /* float [BH, Cq, Ct]     P_T, Eq. 5 */
+    SCOPE_LUT_H,            /* float [BH, Cq, Ch] */
+    SCOPE_LUT_W,            /* float [BH, Cq, Cw] */
+    SCOPE_TOPP_COUNT,       /* int32 [BH, Cq]         t_c, Eq. 7 */
+    SCOPE_BASE_COUNT,       /* int32 [BH, Cq]         b_c, Eq. 8 */
+    SCOPE_K_HEAD,           /* int32 [BH]             Eq. 9 */
+    SCOPE_FINAL_COUNT,      /* int32 [BH, Cq]         r_c, Eq. 10 */
+    SCOPE_KEY_OFFSETS,      /* int64 [BH*Cq + 1]      start of S_c in KEY_INDICES; last = total */
+    SCOPE_KEY_INDICES,      /* int32 [total]          S_c, ascending key index inside a cluster */
+    SCOPE_Q_PERM,           /* int32 [BH, N]          tokens grouped by query cluster, ascending inside */
+    SCOPE_Q_OFFSETS,        /* int32 [BH, Cq + 1]     start of cluster c in Q_PERM (per head) */
+    SCOPE_FIELD_COUNT
+} scope_field;
+
+/* Stages of scope_plan, as bits for scope_plan_stages().  Running a later stage
+ * alone uses whatever the earlier arrays hold (computed or imported). */
+enum {
+    SCOPE_STAGE_KMEANS_INIT = 1,  /* evenly strided initial centroids, u_r = x[floor(r N / C)] */
+    SCOPE_STAGE_KMEANS_Q = 2,     /* kmeans_iters Lloyd iterations on Q (Eq. 2) */
+    SCOPE_STAGE_KMEANS_K = 4,     /* the same on the three key ranges (Eq. 3, Eq. 4) */
+    SCOPE_STAGE_LUT = 8,          /* Eq. 5 */
+    SCOPE_STAGE_SELECT = 16,      /* Eq. 6 - Eq. 10: t_c, b_c, k_head, r_c, key index lists */
+    SCOPE_STAGE_GROUP = 32,       /* query permutation and offsets */
+    SCOPE_STAGE_ALL = 63
+};
+
+/* Bytes of device workspace a plan with these parameters needs (0 if they are invalid). */
+size_t scope_plan_workspace_bytes(const scope_params *params);
+
+/* Validate `params`, lay the plan out inside `workspace` (device pointer, 256-byte
+ * aligned, `bytes` long, caller-owned) and return the host object in *out.  Enqueues
+ * one memset of the status words on `stream`.  Errors: INVALID_ARG, UNSUPPORTED,
+ * ALIGNMENT, WORKSPACE. */
+scope_status scope_plan_create(const scope_params *params, void *workspace, size_t bytes,
+                               void *stream, scope_plan_t **out);
+
+/* Free the host object (never the workspace).  NULL is allowed. */
+void scope_plan_destroy(scope_plan_t *plan);
+
+/* Algorithm 1 lines 1-9: cluster Q and K, build the tables, select the key sets and
+ * group the queries.  Q, K: device, bf16.  Asynchronous on `stream` (a cudaStream_t
+ * passed as void*; NULL is the default stream). */
+scope_status scope_plan(const void *Q, const void *K, scope_plan_t *plan, void *stream);
+
+/* The stages of scope_plan selected by `stages` (SCOPE_STAGE_* bits), in pipeline
+ * order.  Without SCOPE_STAGE_KMEANS_INIT the Lloyd iterations start from the
+ * centroids currently in the plan. */
+scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *plan, uint32_t stages,
+                               void *stream);
+
+/* Eq. 11 (Algorithm 1 lines 10-12): O[Q_c] = softmax(Q[Q_c] K[S_c]^T scale) V[S_c] for
+ * every query cluster of every head, from the plan's Q_PERM/Q_OFFSETS, FINAL_COUNT,
+ * KEY_OFFSETS and KEY_INDICES.  bf16 in, fp32 accumulation, bf16 out.  Every row of O
+ * is written exactly once.  Asynchronous. */
+scope_status scope_sparse_attn(const void *Q, const void *K, const void *V, const scope_plan_t *plan,
+                               void *O, void *stream);
+
+/* scope_plan followed by scope_sparse_attn on the same stream. */
+scope_status scope_forward(const void *Q, const void *K, const void *V, scope_plan_t *plan, void *O,
+                           void *stream);
+
+/* The same layer with HOST tensors (dense [B,H,N,d] bf16; pinned memory makes the
+ * copies asynchronous): copies Q, K, V into `staging` (device, 4*B*H*N*d*2 bytes,
+ * 256-byte aligned, caller-owned), runs scope_forward there and copies O back to
+ * O_host.  Synchronises `stream` before returning. */
+scope_status scope_forward_host(const void *Q_host, const void *K_host, const void *V_host,
+                                scope_plan_t *plan, void *O_host, void *staging, size_t staging_bytes,
+                                void *stream);
+
+/* Dense attention of Eq. 1 through the same attention kernel (every key selected,
+ * identity query grouping); needs no plan arrays, only the plan's shape.  The
+ * comparator of the benchmarks.  Asynchronous. */
+scope_status scope_dense_attn(const void *Q, const void *K, const void *V, const scope_plan_t *plan,
+                              void *O, void *stream);
+
+/* Synchronise `stream` and read the device status word.  Returns SCOPE_OK,
+ * SCOPE_ERR_CAPACITY (then *needed_capacity, if not NULL, receives the number of
+ * index entries the last plan needs), SCOPE_ERR_BAD_PLAN, SCOPE_ERR_TIMEOUT or
+ * SCOPE_ERR_CUDA.  *needed_capacity is also filled on success. */
+scope_status scope_plan_status(const scope_plan_t *plan, void *stream, int64_t *needed_capacity);
+
+/* Clear the device status word (asynchronous).  scope_plan clears it by itself; this is for
+ * flows that import a plan after a failed import or a capacity error. */
+scope_status scope_plan_reset_status(scope_plan_t *plan, void *stream);
+
+/* Device pointer and byte size of a plan array, borrowed from the workspace.  The key
+ * code fields share one packed word per key (T | H << 10 | W << 20) and return that
+ * array for all three. */
+scope_status scope_plan_get(const scope_plan_t *plan, scope_field field, const void **dev_ptr,
+                            size_t *bytes);
+
+/* Bytes scope_plan_export / scope_plan_import move for `field` (0 for a bad field). */
+size_t scope_plan_field_bytes(const scope_plan_t *plan, scope_field field);
+
+/* Copy a plan array to / from HOST memory in the documented shape and type.  Both
+ * synchronise `stream`.  Import checks `bytes` and, for index-bearing fields, value
+ * ranges on the device: a bad array sets the status word to SCOPE_ERR_BAD_PLAN (and
+ * import returns it) instead of being used.  SCOPE_KEY_INDICES moves the first
+ * KEY_OFFSETS[last] entries: import KEY_OFFSETS first. */
+scope_status scope_plan_export(const scope_plan_t *plan, scope_field field, void *host_dst,
+                               size_t bytes, void *stream);
+scope_status scope_plan_import(scope_plan_t *plan, scope_field field, const void *host_src,
+                               size_t bytes, void *stream);
+
+/* Human-readable name of a status code (static string). */
+const char *scope_status_string(scope_status s);
+
+/* k_fix = ceil(alpha N) of Eq. 8 for alpha = alpha_num / alpha_den in exact integer
+ * arithmetic (a float alpha can be off by one).  Returns -1 on bad arguments. */
+int64_t scope_kfix_from_alpha(int64_t N, int64_t alpha_num, int64_t alpha_den);
+
+/* Number of kernels this library has launched in the calling process since load
+ * (diagnostic counter for benchmarks). */
+int64_t scope_kernel_launches(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SCOPE_H */

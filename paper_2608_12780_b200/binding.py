@@ -1,0 +1,271 @@
+"""ctypes binding of libscope_b200.so (the C ABI declared in include/scope.h).
+
+Argument marshalling only: torch provides device memory and the current stream,
+every step of the layer runs in the library's CUDA kernels.  There is no fallback:
+if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libscope_b200.so")
+
+(SCOPE_OK, SCOPE_ERR_INVALID_ARG, SCOPE_ERR_UNSUPPORTED, SCOPE_ERR_ALIGNMENT, SCOPE_ERR_WORKSPACE,
+ SCOPE_ERR_CAPACITY, SCOPE_ERR_BAD_PLAN, SCOPE_ERR_TIMEOUT, SCOPE_ERR_CUDA) = range(9)
+
+FIELDS = ["Q_CENTROIDS", "K_CENTROIDS_T", "K_CENTROIDS_H", "K_CENTROIDS_W", "Q_ASSIGN", "K_CODES_T", "K_CODES_H",
+          "K_CODES_W", "CLUSTER_SIZES", "LUT_T", "LUT_H", "LUT_W", "TOPP_COUNT", "BASE_COUNT", "K_HEAD",
+          "FINAL_COUNT", "KEY_OFFSETS", "KEY_INDICES", "Q_PERM", "Q_OFFSETS"]
+FIELD_ID = {n: i for i, n in enumerate(FIELDS)}
+_FLOAT_FIELDS = {"Q_CENTROIDS", "K_CENTROIDS_T", "K_CENTROIDS_H", "K_CENTROIDS_W", "LUT_T", "LUT_H", "LUT_W"}
+
+STAGE_KMEANS_INIT, STAGE_KMEANS_Q, STAGE_KMEANS_K, STAGE_LUT, STAGE_SELECT, STAGE_GROUP = 1, 2, 4, 8, 16, 32
+STAGE_ALL = 63
+
+EXPORTS = ["scope_plan_workspace_bytes", "scope_plan_create", "scope_plan_destroy", "scope_plan", "scope_plan_stages",
+           "scope_sparse_attn", "scope_forward", "scope_forward_host", "scope_dense_attn", "scope_plan_status",
+           "scope_plan_reset_status", "scope_plan_get", "scope_plan_field_bytes", "scope_plan_export",
+           "scope_plan_import", "scope_status_string", "scope_kfix_from_alpha", "scope_kernel_launches"]
+
+
+class ScopeParams(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("N", C.c_int32), ("d", C.c_int32),
+                ("d_t", C.c_int32), ("d_h", C.c_int32), ("d_w", C.c_int32),
+                ("Cq", C.c_int32), ("Ct", C.c_int32), ("Ch", C.c_int32), ("Cw", C.c_int32),
+                ("kmeans_iters", C.c_int32), ("top_p", C.c_float), ("k_fix", C.c_int32), ("scale", C.c_float),
+                ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_n", C.c_int64),
+                ("index_capacity", C.c_int64)]
+
+
+class ScopeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2608_12780_b200.build` "
+                               "(there is no CPU or PyTorch fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, sz, i64 = C.c_void_p, C.c_size_t, C.c_int64
+        PP = C.POINTER(ScopeParams)
+        L.scope_plan_workspace_bytes.argtypes = [PP]
+        L.scope_plan_workspace_bytes.restype = sz
+        L.scope_plan_create.argtypes = [PP, vp, sz, vp, C.POINTER(vp)]
+        L.scope_plan_destroy.argtypes = [vp]
+        L.scope_plan_destroy.restype = None
+        L.scope_plan.argtypes = [vp, vp, vp, vp]
+        L.scope_plan_stages.argtypes = [vp, vp, vp, C.c_uint32, vp]
+        L.scope_sparse_attn.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.scope_dense_attn.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.scope_forward.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.scope_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+        L.scope_plan_status.argtypes = [vp, vp, C.POINTER(i64)]
+        L.scope_plan_reset_status.argtypes = [vp, vp]
+        L.scope_plan_get.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(sz)]
+        L.scope_plan_field_bytes.argtypes = [vp, C.c_int]
+        L.scope_plan_field_bytes.restype = sz
+        L.scope_plan_export.argtypes = [vp, C.c_int, vp, sz, vp]
+        L.scope_plan_import.argtypes = [vp, C.c_int, vp, sz, vp]
+        L.scope_status_string.argtypes = [C.c_int]
+        L.scope_status_string.restype = C.c_char_p
+        L.scope_kfix_from_alpha.argtypes = [i64, i64, i64]
+        L.scope_kfix_from_alpha.restype = i64
+        L.scope_kernel_launches.argtypes = []
+        L.scope_kernel_launches.restype = i64
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().scope_status_string(int(status)).decode()
+
+
+def scope_kfix_from_alpha(N: int, alpha_num: int, alpha_den: int) -> int:
+    return int(lib().scope_kfix_from_alpha(N, alpha_num, alpha_den))
+
+
+def scope_kernel_launches() -> int:
+    return int(lib().scope_kernel_launches())
+
+
+def _check(status: int, where: str):
+    if status != SCOPE_OK:
+        raise ScopeError(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def make_params(cfg, B=None, H=None, index_capacity=None, strides=(0, 0, 0), scale=None) -> ScopeParams:
+    """ScopeParams from a config object with grid/split/Cq/... attributes (see inputs.ScopeConfig)."""
+    B = cfg.B if B is None else B
+    H = cfg.H if H is None else H
+    N = cfg.N
+    if index_capacity is None:
+        index_capacity = max(1, int(0.35 * B * H * cfg.Cq * N))
+    return ScopeParams(B, H, N, cfg.d, cfg.split[0], cfg.split[1], cfg.split[2], cfg.Cq, cfg.Ct, cfg.Ch, cfg.Cw,
+                       cfg.iters, cfg.top_p, cfg.k_fix, cfg.scale if scale is None else scale,
+                       strides[0], strides[1], strides[2], int(index_capacity))
+
+
+def _dev_ptr(t: torch.Tensor, name: str) -> int:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.bfloat16):
+        raise TypeError(f"{name} must be a CUDA bfloat16 tensor")
+    return t.data_ptr()
+
+
+class Plan:
+    """A scope_plan_t plus the torch-allocated workspace it lives in."""
+
+    def __init__(self, params: ScopeParams, device="cuda"):
+        L = lib()
+        self.params = params
+        nbytes = L.scope_plan_workspace_bytes(C.byref(params))
+        if nbytes == 0:
+            # let scope_plan_create name the reason
+            h = C.c_void_p()
+            _check(L.scope_plan_create(C.byref(params), C.c_void_p(256), 0, None, C.byref(h)), "scope_plan_create")
+            raise ScopeError(SCOPE_ERR_INVALID_ARG, "scope_plan_workspace_bytes")
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+        base = (self.workspace.data_ptr() + 255) & ~255
+        h = C.c_void_p()
+        _check(L.scope_plan_create(C.byref(params), C.c_void_p(base), nbytes, C.c_void_p(_stream()), C.byref(h)),
+               "scope_plan_create")
+        self.handle = h
+        self.workspace_bytes = nbytes
+
+    def __del__(self):
+        h = getattr(self, "handle", None)
+        if h is not None and _lib is not None:
+            _lib.scope_plan_destroy(h)
+            self.handle = None
+
+    # ---- shape helpers
+    @property
+    def BH(self):
+        return self.params.B * self.params.H
+
+    def field_shape(self, name: str):
+        p, BH = self.params, self.BH
+        return {
+            "Q_CENTROIDS": (BH, p.Cq, p.d), "K_CENTROIDS_T": (BH, p.Ct, p.d_t), "K_CENTROIDS_H": (BH, p.Ch, p.d_h),
+            "K_CENTROIDS_W": (BH, p.Cw, p.d_w), "Q_ASSIGN": (BH, p.N), "K_CODES_T": (BH, p.N), "K_CODES_H": (BH, p.N),
+            "K_CODES_W": (BH, p.N), "CLUSTER_SIZES": (BH, p.Cq), "LUT_T": (BH, p.Cq, p.Ct), "LUT_H": (BH, p.Cq, p.Ch),
+            "LUT_W": (BH, p.Cq, p.Cw), "TOPP_COUNT": (BH, p.Cq), "BASE_COUNT": (BH, p.Cq), "K_HEAD": (BH,),
+            "FINAL_COUNT": (BH, p.Cq), "KEY_OFFSETS": (BH * p.Cq + 1,), "Q_PERM": (BH, p.N), "Q_OFFSETS": (BH, p.Cq + 1),
+        }[name]
+
+    # ---- calls
+    def status(self):
+        need = C.c_int64(0)
+        s = lib().scope_plan_status(self.handle, C.c_void_p(_stream()), C.byref(need))
+        return int(s), int(need.value)
+
+    def check(self, where="scope_plan_status"):
+        s, need = self.status()
+        if s == SCOPE_ERR_CAPACITY:
+            raise ScopeError(s, f"{where} (needed capacity {need}, have {self.params.index_capacity})")
+        _check(s, where)
+        return need
+
+    def reset_status(self):
+        _check(lib().scope_plan_reset_status(self.handle, C.c_void_p(_stream())), "scope_plan_reset_status")
+
+    def export(self, name: str) -> np.ndarray:
+        fid = FIELD_ID[name]
+        if name == "KEY_INDICES":
+            total = int(self.export("KEY_OFFSETS")[-1])
+            out = np.empty(total, np.int32)
+        else:
+            dt = np.float32 if name in _FLOAT_FIELDS else (np.int64 if name == "KEY_OFFSETS" else np.int32)
+            out = np.empty(self.field_shape(name), dt)
+        _check(lib().scope_plan_export(self.handle, fid, out.ctypes.data_as(C.c_void_p), out.nbytes,
+                                       C.c_void_p(_stream())), f"scope_plan_export({name})")
+        return out
+
+    def import_(self, name: str, arr) -> None:
+        fid = FIELD_ID[name]
+        dt = np.float32 if name in _FLOAT_FIELDS else (np.int64 if name == "KEY_OFFSETS" else np.int32)
+        a = np.ascontiguousarray(arr, dtype=dt)
+        _check(lib().scope_plan_import(self.handle, fid, a.ctypes.data_as(C.c_void_p), a.nbytes,
+                                       C.c_void_p(_stream())), f"scope_plan_import({name})")
+
+    def get(self, name: str):
+        ptr, nb = C.c_void_p(), C.c_size_t()
+        _check(lib().scope_plan_get(self.handle, FIELD_ID[name], C.byref(ptr), C.byref(nb)), "scope_plan_get")
+        return int(ptr.value), int(nb.value)
+
+
+def scope_plan_create(params: ScopeParams, device="cuda") -> Plan:
+    return Plan(params, device)
+
+
+def scope_plan(Q, K, plan: Plan) -> None:
+    """Algorithm 1 lines 1-9 on the current stream (asynchronous)."""
+    _check(lib().scope_plan(_dev_ptr(Q, "Q"), _dev_ptr(K, "K"), plan.handle, C.c_void_p(_stream())), "scope_plan")
+
+
+def scope_plan_stages(Q, K, plan: Plan, stages: int) -> None:
+    q = _dev_ptr(Q, "Q") if Q is not None else None
+    k = _dev_ptr(K, "K") if K is not None else None
+    _check(lib().scope_plan_stages(q, k, plan.handle, stages, C.c_void_p(_stream())), "scope_plan_stages")
+
+
+def scope_sparse_attn(Q, K, V, plan: Plan, O=None):
+    """Eq. 11 on the current stream; returns O (bf16, same layout as Q)."""
+    if O is None:
+        O = torch.empty_like(Q)
+    _check(lib().scope_sparse_attn(_dev_ptr(Q, "Q"), _dev_ptr(K, "K"), _dev_ptr(V, "V"), plan.handle,
+                                   _dev_ptr(O, "O"), C.c_void_p(_stream())), "scope_sparse_attn")
+    return O
+
+
+def scope_dense_attn(Q, K, V, plan: Plan, O=None):
+    """Eq. 1 through the same kernel."""
+    if O is None:
+        O = torch.empty_like(Q)
+    _check(lib().scope_dense_attn(_dev_ptr(Q, "Q"), _dev_ptr(K, "K"), _dev_ptr(V, "V"), plan.handle,
+                                  _dev_ptr(O, "O"), C.c_void_p(_stream())), "scope_dense_attn")
+    return O
+
+
+def scope_forward(Q, K, V, plan: Plan, O=None):
+    """scope_plan + scope_sparse_attn on the current stream."""
+    if O is None:
+        O = torch.empty_like(Q)
+    _check(lib().scope_forward(_dev_ptr(Q, "Q"), _dev_ptr(K, "K"), _dev_ptr(V, "V"), plan.handle,
+                               _dev_ptr(O, "O"), C.c_void_p(_stream())), "scope_forward")
+    return O
+
+
+def scope_forward_host(Qh, Kh, Vh, plan: Plan, Oh, staging: torch.Tensor) -> None:
+    """The layer on HOST tensors (torch CPU bf16, ideally pinned); synchronous."""
+    for t in (Qh, Kh, Vh, Oh):
+        if t.is_cuda or t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise TypeError("host tensors must be contiguous CPU bfloat16")
+    base = (staging.data_ptr() + 255) & ~255
+    nbytes = staging.numel() * staging.element_size() - (base - staging.data_ptr())
+    _check(lib().scope_forward_host(Qh.data_ptr(), Kh.data_ptr(), Vh.data_ptr(), plan.handle, Oh.data_ptr(),
+                                    C.c_void_p(base), nbytes, C.c_void_p(_stream())), "scope_forward_host")
+
+
+def bits_to_torch(u16: np.ndarray, device=None, pin=False) -> torch.Tensor:
+    """uint16 bf16 bit patterns -> torch bfloat16 tensor (no value conversion)."""
+    t = torch.from_numpy(u16.view(np.int16)).view(torch.bfloat16)
+    if pin:
+        t = t.pin_memory()
+    return t.to(device, non_blocking=pin) if device is not None else t

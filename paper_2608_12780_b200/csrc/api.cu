@@ -1,0 +1,591 @@
+// C ABI of the library: parameter validation, workspace layout, stage sequencing, plan import /
+// export.  All device work is enqueued by the launchers of the kernel files.
+#include <atomic>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "scope_internal.cuh"
+
+using namespace scope;
+
+struct scope_plan_s {
+    scope_params p;
+    int BH;
+    unsigned char *ws;
+    size_t ws_bytes;
+    int32_t *status;
+    // plan arrays
+    float *q_cent, *k_cent[3];
+    int32_t *q_assign;
+    uint32_t *k_codes;
+    int32_t *n_c;
+    float *lut[3];
+    int32_t *t_c, *b_c, *r_c, *k_head;
+    int64_t *key_offsets;
+    int32_t *key_indices;
+    int32_t *q_perm, *q_offsets;
+    // scratch
+    float *q_unorm, *k_unorm[3], *q_u2max, *k_u2max[3];
+    double *q_sums, *k_sums[3];
+    int32_t *q_counts, *k_counts[3];
+    RowState *rows;
+    int32_t *tile_offsets;
+    int32_t *io_scratch;  // [BH, N] staging for packed-code import / export
+};
+
+namespace scope {
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace scope
+
+namespace {
+
+struct Carver {
+    unsigned char *base;
+    size_t off = 0;
+    template <typename T>
+    T *take(size_t n)
+    {
+        off = (off + 255) & ~(size_t)255;
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+};
+
+scope_status validate(const scope_params *p)
+{
+    if (!p)
+        return SCOPE_ERR_INVALID_ARG;
+    if (p->B < 1 || p->H < 1 || p->N < 1 || p->d < 1)
+        return SCOPE_ERR_INVALID_ARG;
+    if (p->d != kHeadDim)
+        return SCOPE_ERR_UNSUPPORTED;
+    if (p->d_t < 1 || p->d_h < 1 || p->d_w < 1 || p->d_t + p->d_h + p->d_w != p->d)
+        return SCOPE_ERR_INVALID_ARG;
+    const int32_t cs[4] = {p->Cq, p->Ct, p->Ch, p->Cw};
+    for (int c : cs) {
+        if (c < 1 || c > p->N)
+            return SCOPE_ERR_INVALID_ARG;
+        if (c > kMaxClusters)
+            return SCOPE_ERR_UNSUPPORTED;
+    }
+    if (p->kmeans_iters < 1)
+        return SCOPE_ERR_INVALID_ARG;
+    if (!(p->top_p > 0.f) || !std::isfinite(p->top_p))
+        return SCOPE_ERR_INVALID_ARG;
+    if (p->k_fix < 1 || p->k_fix > p->N)
+        return SCOPE_ERR_INVALID_ARG;
+    if (p->scale < 0.f || !std::isfinite(p->scale))
+        return SCOPE_ERR_INVALID_ARG;
+    if (p->index_capacity < 1)
+        return SCOPE_ERR_INVALID_ARG;
+    const bool dense = p->stride_b == 0 && p->stride_h == 0 && p->stride_n == 0;
+    if (!dense) {
+        if (p->stride_n < p->d || p->stride_h < 1 || p->stride_b < 1)
+            return SCOPE_ERR_INVALID_ARG;
+        if (p->stride_n % 8 || p->stride_h % 8 || p->stride_b % 8)
+            return SCOPE_ERR_ALIGNMENT;
+    }
+    if ((int64_t)p->B * p->H * (int64_t)p->Cq > (int64_t)1 << 30)
+        return SCOPE_ERR_UNSUPPORTED;
+    return SCOPE_OK;
+}
+
+void carve(scope_plan_t *pl, unsigned char *base, size_t *total)
+{
+    const scope_params &p = pl->p;
+    const size_t BH = (size_t)p.B * p.H, N = p.N, Cq = p.Cq;
+    const size_t C[3] = {(size_t)p.Ct, (size_t)p.Ch, (size_t)p.Cw}, D[3] = {(size_t)p.d_t, (size_t)p.d_h, (size_t)p.d_w};
+    Carver cv{base};
+    pl->status = cv.take<int32_t>(ST_WORDS);
+    pl->q_cent = cv.take<float>(BH * Cq * p.d);
+    pl->q_unorm = cv.take<float>(BH * Cq);
+    pl->q_u2max = cv.take<float>(BH);
+    pl->q_sums = cv.take<double>(BH * Cq * p.d);
+    pl->q_counts = cv.take<int32_t>(BH * Cq);
+    for (int m = 0; m < 3; ++m) {
+        pl->k_cent[m] = cv.take<float>(BH * C[m] * D[m]);
+        pl->k_unorm[m] = cv.take<float>(BH * C[m]);
+        pl->k_u2max[m] = cv.take<float>(BH);
+        pl->k_sums[m] = cv.take<double>(BH * C[m] * D[m]);
+        pl->k_counts[m] = cv.take<int32_t>(BH * C[m]);
+        pl->lut[m] = cv.take<float>(BH * Cq * C[m]);
+    }
+    pl->q_assign = cv.take<int32_t>(BH * N);
+    pl->k_codes = cv.take<uint32_t>(BH * N);
+    pl->n_c = cv.take<int32_t>(BH * Cq);
+    pl->t_c = cv.take<int32_t>(BH * Cq);
+    pl->b_c = cv.take<int32_t>(BH * Cq);
+    pl->r_c = cv.take<int32_t>(BH * Cq);
+    pl->k_head = cv.take<int32_t>(BH);
+    pl->rows = cv.take<RowState>(BH * Cq);
+    pl->key_offsets = cv.take<int64_t>(BH * Cq + 1);
+    pl->q_perm = cv.take<int32_t>(BH * N);
+    pl->q_offsets = cv.take<int32_t>(BH * (Cq + 1));
+    pl->tile_offsets = cv.take<int32_t>(BH * (Cq + 1));
+    pl->io_scratch = cv.take<int32_t>(BH * N);
+    pl->key_indices = cv.take<int32_t>((size_t)p.index_capacity);
+    *total = (cv.off + 255) & ~(size_t)255;
+}
+
+void normalise(scope_params *p)
+{
+    if (p->stride_b == 0 && p->stride_h == 0 && p->stride_n == 0) {
+        p->stride_n = p->d;
+        p->stride_h = (int64_t)p->N * p->d;
+        p->stride_b = (int64_t)p->H * p->N * p->d;
+    }
+    if (p->scale == 0.f)
+        p->scale = 1.0f / sqrtf((float)p->d);
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+KmArgs q_args(const scope_plan_t *pl, const void *Q)
+{
+    KmArgs a{};
+    const scope_params &p = pl->p;
+    a.X = static_cast<const bf16 *>(Q);
+    a.sb = p.stride_b; a.sh = p.stride_h; a.sn = p.stride_n;
+    a.B = p.B; a.H = p.H; a.N = p.N;
+    a.nspaces = 1;
+    a.sp[0] = KmSpace{0, p.d, p.Cq, pl->q_cent, pl->q_unorm, pl->q_u2max, pl->q_sums, pl->q_counts, pl->n_c};
+    a.assign = pl->q_assign;
+    a.codes = nullptr;
+    return a;
+}
+
+KmArgs k_args(const scope_plan_t *pl, const void *K)
+{
+    KmArgs a{};
+    const scope_params &p = pl->p;
+    a.X = static_cast<const bf16 *>(K);
+    a.sb = p.stride_b; a.sh = p.stride_h; a.sn = p.stride_n;
+    a.B = p.B; a.H = p.H; a.N = p.N;
+    a.nspaces = 3;
+    const int ch0[3] = {0, p.d_t, p.d_t + p.d_h}, D[3] = {p.d_t, p.d_h, p.d_w}, C[3] = {p.Ct, p.Ch, p.Cw};
+    for (int m = 0; m < 3; ++m)
+        a.sp[m] = KmSpace{ch0[m], D[m], C[m], pl->k_cent[m], pl->k_unorm[m], pl->k_u2max[m], pl->k_sums[m],
+                          pl->k_counts[m], nullptr};
+    a.assign = nullptr;
+    a.codes = pl->k_codes;
+    return a;
+}
+
+AttnArgs attn_args(const scope_plan_t *pl, const void *Q, const void *K, const void *V, void *O, int dense)
+{
+    const scope_params &p = pl->p;
+    AttnArgs a{};
+    a.Q = static_cast<const bf16 *>(Q);
+    a.K = static_cast<const bf16 *>(K);
+    a.V = static_cast<const bf16 *>(V);
+    a.O = static_cast<bf16 *>(O);
+    a.sb = p.stride_b; a.sh = p.stride_h; a.sn = p.stride_n;
+    a.B = p.B; a.H = p.H; a.N = p.N; a.Cq = p.Cq;
+    a.scale = p.scale;
+    a.dense = dense;
+    a.q_perm = pl->q_perm; a.q_offsets = pl->q_offsets; a.tile_offsets = pl->tile_offsets;
+    a.r_c = pl->r_c; a.key_offsets = pl->key_offsets; a.key_indices = pl->key_indices;
+    a.status = pl->status;
+    const int full = (p.N + kAttnTileRows - 1) / kAttnTileRows;
+    a.max_tiles_per_head = dense ? full : (int)std::min<int64_t>((int64_t)p.N, (int64_t)p.N / kAttnTileRows + p.Cq);
+    return a;
+}
+
+scope_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? SCOPE_OK : SCOPE_ERR_CUDA; }
+
+struct FieldInfo {
+    void *ptr;
+    size_t elems;
+    size_t elem_bytes;
+    int code_field;  // 0..2 for packed key codes, -1 otherwise
+};
+
+bool field_info(const scope_plan_t *pl, scope_field f, FieldInfo *out)
+{
+    const scope_params &p = pl->p;
+    const size_t BH = pl->BH, N = p.N, Cq = p.Cq;
+    FieldInfo fi{nullptr, 0, 4, -1};
+    switch (f) {
+    case SCOPE_Q_CENTROIDS: fi = {pl->q_cent, BH * Cq * p.d, 4, -1}; break;
+    case SCOPE_K_CENTROIDS_T: fi = {pl->k_cent[0], BH * p.Ct * p.d_t, 4, -1}; break;
+    case SCOPE_K_CENTROIDS_H: fi = {pl->k_cent[1], BH * p.Ch * p.d_h, 4, -1}; break;
+    case SCOPE_K_CENTROIDS_W: fi = {pl->k_cent[2], BH * p.Cw * p.d_w, 4, -1}; break;
+    case SCOPE_Q_ASSIGN: fi = {pl->q_assign, BH * N, 4, -1}; break;
+    case SCOPE_K_CODES_T: fi = {pl->k_codes, BH * N, 4, 0}; break;
+    case SCOPE_K_CODES_H: fi = {pl->k_codes, BH * N, 4, 1}; break;
+    case SCOPE_K_CODES_W: fi = {pl->k_codes, BH * N, 4, 2}; break;
+    case SCOPE_CLUSTER_SIZES: fi = {pl->n_c, BH * Cq, 4, -1}; break;
+    case SCOPE_LUT_T: fi = {pl->lut[0], BH * Cq * p.Ct, 4, -1}; break;
+    case SCOPE_LUT_H: fi = {pl->lut[1], BH * Cq * p.Ch, 4, -1}; break;
+    case SCOPE_LUT_W: fi = {pl->lut[2], BH * Cq * p.Cw, 4, -1}; break;
+    case SCOPE_TOPP_COUNT: fi = {pl->t_c, BH * Cq, 4, -1}; break;
+    case SCOPE_BASE_COUNT: fi = {pl->b_c, BH * Cq, 4, -1}; break;
+    case SCOPE_K_HEAD: fi = {pl->k_head, BH, 4, -1}; break;
+    case SCOPE_FINAL_COUNT: fi = {pl->r_c, BH * Cq, 4, -1}; break;
+    case SCOPE_KEY_OFFSETS: fi = {pl->key_offsets, BH * Cq + 1, 8, -1}; break;
+    case SCOPE_KEY_INDICES: fi = {pl->key_indices, (size_t)p.index_capacity, 4, -1}; break;
+    case SCOPE_Q_PERM: fi = {pl->q_perm, BH * N, 4, -1}; break;
+    case SCOPE_Q_OFFSETS: fi = {pl->q_offsets, BH * (Cq + 1), 4, -1}; break;
+    default: return false;
+    }
+    *out = fi;
+    return true;
+}
+
+// entries of KEY_INDICES in use = KEY_OFFSETS[last]; synchronises the stream
+scope_status indices_in_use(const scope_plan_t *pl, cudaStream_t st, int64_t *n)
+{
+    int64_t total = 0;
+    cudaError_t e = cudaMemcpyAsync(&total, pl->key_offsets + (size_t)pl->BH * pl->p.Cq, sizeof total,
+                                    cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess)
+        e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess)
+        return SCOPE_ERR_CUDA;
+    if (total < 0 || total > pl->p.index_capacity)
+        return SCOPE_ERR_BAD_PLAN;
+    *n = total;
+    return SCOPE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t scope_plan_workspace_bytes(const scope_params *params)
+{
+    if (validate(params) != SCOPE_OK)
+        return 0;
+    scope_plan_t tmp{};
+    tmp.p = *params;
+    normalise(&tmp.p);
+    size_t total = 0;
+    carve(&tmp, nullptr, &total);
+    return total;
+}
+
+scope_status scope_plan_create(const scope_params *params, void *workspace, size_t bytes, void *stream,
+                               scope_plan_t **out)
+{
+    if (!out)
+        return SCOPE_ERR_INVALID_ARG;
+    *out = nullptr;
+    scope_status s = validate(params);
+    if (s != SCOPE_OK)
+        return s;
+    if (!workspace)
+        return SCOPE_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u)
+        return SCOPE_ERR_ALIGNMENT;
+    scope_plan_t *pl = new (std::nothrow) scope_plan_t{};
+    if (!pl)
+        return SCOPE_ERR_INVALID_ARG;
+    pl->p = *params;
+    normalise(&pl->p);
+    pl->BH = pl->p.B * pl->p.H;
+    size_t total = 0;
+    carve(pl, static_cast<unsigned char *>(workspace), &total);
+    if (bytes < total) {
+        delete pl;
+        return SCOPE_ERR_WORKSPACE;
+    }
+    pl->ws = static_cast<unsigned char *>(workspace);
+    pl->ws_bytes = bytes;
+    if (cudaMemsetAsync(pl->status, 0, ST_WORDS * sizeof(int32_t), static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        delete pl;
+        return SCOPE_ERR_CUDA;
+    }
+    *out = pl;
+    return SCOPE_OK;
+}
+
+void scope_plan_destroy(scope_plan_t *plan) { delete plan; }
+
+scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, uint32_t stages, void *stream)
+{
+    if (!pl || (stages & ~(uint32_t)SCOPE_STAGE_ALL))
+        return SCOPE_ERR_INVALID_ARG;
+    const bool needQ = stages & (SCOPE_STAGE_KMEANS_INIT | SCOPE_STAGE_KMEANS_Q);
+    const bool needK = stages & (SCOPE_STAGE_KMEANS_INIT | SCOPE_STAGE_KMEANS_K);
+    if ((needQ && !Q) || (needK && !K))
+        return SCOPE_ERR_INVALID_ARG;
+    if ((needQ && !aligned16(Q)) || (needK && !aligned16(K)))
+        return SCOPE_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const scope_params &p = pl->p;
+
+    if (stages & SCOPE_STAGE_SELECT) {
+        // a fresh selection clears an earlier capacity verdict
+        if (cudaMemsetAsync(pl->status, 0, ST_WORDS * sizeof(int32_t), st) != cudaSuccess)
+            return SCOPE_ERR_CUDA;
+    }
+    if (stages & SCOPE_STAGE_KMEANS_INIT) {
+        launch_kmeans_init(q_args(pl, Q), st);
+        launch_kmeans_init(k_args(pl, K), st);
+    }
+    if (stages & SCOPE_STAGE_KMEANS_Q) {
+        KmArgs a = q_args(pl, Q);
+        if (!(stages & SCOPE_STAGE_KMEANS_INIT))
+            launch_kmeans_norms(a, st);  // centroids may have been imported
+        for (int it = 0; it < p.kmeans_iters; ++it)
+            launch_kmeans_iteration(a, st);
+    }
+    if (stages & SCOPE_STAGE_KMEANS_K) {
+        KmArgs a = k_args(pl, K);
+        if (!(stages & SCOPE_STAGE_KMEANS_INIT))
+            launch_kmeans_norms(a, st);
+        for (int it = 0; it < p.kmeans_iters; ++it)
+            launch_kmeans_iteration(a, st);
+    }
+    if (stages & SCOPE_STAGE_LUT) {
+        KmArgs a = k_args(pl, K);
+        launch_lut(pl->BH, p.Cq, p.d, pl->q_cent, a.sp, pl->lut, st);
+    }
+    if (stages & SCOPE_STAGE_SELECT) {
+        SelectArgs a{};
+        a.BH = pl->BH; a.N = p.N; a.Cq = p.Cq; a.Ct = p.Ct; a.Ch = p.Ch; a.Cw = p.Cw;
+        a.scale = p.scale; a.top_p = p.top_p; a.k_fix = p.k_fix; a.capacity = p.index_capacity;
+        a.codes = pl->k_codes;
+        a.lutT = pl->lut[0]; a.lutH = pl->lut[1]; a.lutW = pl->lut[2];
+        a.n_c = pl->n_c;
+        a.t_c = pl->t_c; a.b_c = pl->b_c; a.r_c = pl->r_c; a.k_head = pl->k_head;
+        a.rows = pl->rows;
+        a.key_offsets = pl->key_offsets; a.key_indices = pl->key_indices;
+        a.status = pl->status;
+        launch_select(a, st);
+    }
+    if (stages & SCOPE_STAGE_GROUP) {
+        GroupArgs a{};
+        a.BH = pl->BH; a.N = p.N; a.Cq = p.Cq;
+        a.g = pl->q_assign; a.n_c = pl->n_c;
+        a.q_perm = pl->q_perm; a.q_offsets = pl->q_offsets; a.tile_offsets = pl->tile_offsets;
+        a.tile_rows = kAttnTileRows;
+        launch_group(a, st);
+    }
+    return cuda_ok(cudaGetLastError());
+}
+
+scope_status scope_plan(const void *Q, const void *K, scope_plan_t *plan, void *stream)
+{
+    return scope_plan_stages(Q, K, plan, SCOPE_STAGE_ALL, stream);
+}
+
+static scope_status attn_common(const void *Q, const void *K, const void *V, const scope_plan_t *pl, void *O,
+                                void *stream, int dense)
+{
+    if (!pl || !Q || !K || !V || !O)
+        return SCOPE_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O))
+        return SCOPE_ERR_ALIGNMENT;
+    launch_attn(attn_args(pl, Q, K, V, O, dense), static_cast<cudaStream_t>(stream));
+    return cuda_ok(cudaGetLastError());
+}
+
+scope_status scope_sparse_attn(const void *Q, const void *K, const void *V, const scope_plan_t *plan, void *O,
+                               void *stream)
+{
+    return attn_common(Q, K, V, plan, O, stream, 0);
+}
+
+scope_status scope_dense_attn(const void *Q, const void *K, const void *V, const scope_plan_t *plan, void *O,
+                              void *stream)
+{
+    return attn_common(Q, K, V, plan, O, stream, 1);
+}
+
+scope_status scope_forward(const void *Q, const void *K, const void *V, scope_plan_t *plan, void *O, void *stream)
+{
+    if (!plan || !Q || !K || !V || !O)
+        return SCOPE_ERR_INVALID_ARG;
+    scope_status s = scope_plan(Q, K, plan, stream);
+    if (s != SCOPE_OK)
+        return s;
+    return scope_sparse_attn(Q, K, V, plan, O, stream);
+}
+
+scope_status scope_forward_host(const void *Qh, const void *Kh, const void *Vh, scope_plan_t *pl, void *Oh,
+                                void *staging, size_t staging_bytes, void *stream)
+{
+    if (!pl || !Qh || !Kh || !Vh || !Oh || !staging)
+        return SCOPE_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(staging) & 255u)
+        return SCOPE_ERR_ALIGNMENT;
+    scope_params &p = pl->p;
+    const size_t one = (size_t)p.B * p.H * p.N * p.d * sizeof(bf16);
+    if (staging_bytes < 4 * one)
+        return SCOPE_ERR_WORKSPACE;
+    if (p.stride_n != p.d || p.stride_h != (int64_t)p.N * p.d || p.stride_b != (int64_t)p.H * p.N * p.d)
+        return SCOPE_ERR_UNSUPPORTED;  // host tensors are dense
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char *dev = static_cast<unsigned char *>(staging);
+    void *dQ = dev, *dK = dev + one, *dV = dev + 2 * one, *dO = dev + 3 * one;
+    if (cudaMemcpyAsync(dQ, Qh, one, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dK, Kh, one, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dV, Vh, one, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return SCOPE_ERR_CUDA;
+    scope_status s = scope_forward(dQ, dK, dV, pl, dO, stream);
+    if (s != SCOPE_OK)
+        return s;
+    if (cudaMemcpyAsync(Oh, dO, one, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return SCOPE_ERR_CUDA;
+    return scope_plan_status(pl, stream, nullptr);
+}
+
+scope_status scope_plan_status(const scope_plan_t *pl, void *stream, int64_t *needed_capacity)
+{
+    if (!pl)
+        return SCOPE_ERR_INVALID_ARG;
+    int32_t host[4] = {0, 0, 0, 0};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(host, pl->status, sizeof host, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess)
+        e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess)
+        return SCOPE_ERR_CUDA;
+    if (needed_capacity) {
+        int64_t v;
+        std::memcpy(&v, host + ST_NEEDED_LO, sizeof v);
+        *needed_capacity = v;
+    }
+    if (host[ST_CODE] < 0 || host[ST_CODE] > SCOPE_ERR_CUDA)
+        return SCOPE_ERR_CUDA;
+    return static_cast<scope_status>(host[ST_CODE]);
+}
+
+scope_status scope_plan_reset_status(scope_plan_t *pl, void *stream)
+{
+    if (!pl)
+        return SCOPE_ERR_INVALID_ARG;
+    return cuda_ok(cudaMemsetAsync(pl->status, 0, ST_WORDS * sizeof(int32_t), static_cast<cudaStream_t>(stream)));
+}
+
+scope_status scope_plan_get(const scope_plan_t *pl, scope_field field, const void **dev_ptr, size_t *bytes)
+{
+    FieldInfo fi;
+    if (!pl || !dev_ptr || !field_info(pl, field, &fi))
+        return SCOPE_ERR_INVALID_ARG;
+    *dev_ptr = fi.ptr;
+    if (bytes)
+        *bytes = fi.elems * fi.elem_bytes;
+    return SCOPE_OK;
+}
+
+size_t scope_plan_field_bytes(const scope_plan_t *pl, scope_field field)
+{
+    FieldInfo fi;
+    if (!pl || !field_info(pl, field, &fi))
+        return 0;
+    return fi.elems * fi.elem_bytes;
+}
+
+scope_status scope_plan_export(const scope_plan_t *pl, scope_field field, void *host_dst, size_t bytes, void *stream)
+{
+    FieldInfo fi;
+    if (!pl || !host_dst || !field_info(pl, field, &fi))
+        return SCOPE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    size_t want = fi.elems * fi.elem_bytes;
+    if (field == SCOPE_KEY_INDICES) {
+        int64_t used = 0;
+        scope_status s = indices_in_use(pl, st, &used);
+        if (s != SCOPE_OK)
+            return s;
+        want = (size_t)used * 4;
+        if (bytes < want)
+            return SCOPE_ERR_INVALID_ARG;
+    } else if (bytes != want) {
+        return SCOPE_ERR_INVALID_ARG;
+    }
+    const void *src = fi.ptr;
+    if (fi.code_field >= 0) {
+        launch_unpack_codes(pl->k_codes, pl->io_scratch, (int64_t)fi.elems, fi.code_field, st);
+        src = pl->io_scratch;
+    }
+    cudaError_t e = want ? cudaMemcpyAsync(host_dst, src, want, cudaMemcpyDeviceToHost, st) : cudaSuccess;
+    if (e == cudaSuccess)
+        e = cudaStreamSynchronize(st);
+    return cuda_ok(e);
+}
+
+scope_status scope_plan_import(scope_plan_t *pl, scope_field field, const void *host_src, size_t bytes, void *stream)
+{
+    FieldInfo fi;
+    if (!pl || !host_src || !field_info(pl, field, &fi))
+        return SCOPE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const scope_params &p = pl->p;
+    size_t want = fi.elems * fi.elem_bytes;
+    if (field == SCOPE_KEY_INDICES) {
+        int64_t used = 0;
+        scope_status s = indices_in_use(pl, st, &used);
+        if (s != SCOPE_OK)
+            return s;
+        want = (size_t)used * 4;
+    }
+    if (bytes != want)
+        return SCOPE_ERR_INVALID_ARG;
+    void *dst = fi.code_field >= 0 ? static_cast<void *>(pl->io_scratch) : fi.ptr;
+    if (want && cudaMemcpyAsync(dst, host_src, want, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return SCOPE_ERR_CUDA;
+    const int64_t n = (int64_t)(want / fi.elem_bytes);
+    const int Cm[3] = {p.Ct, p.Ch, p.Cw};
+    switch (field) {
+    case SCOPE_Q_ASSIGN: launch_check_range_i32(pl->q_assign, n, 0, p.Cq - 1, pl->status, st); break;
+    case SCOPE_K_CODES_T:
+    case SCOPE_K_CODES_H:
+    case SCOPE_K_CODES_W:
+        launch_pack_codes(pl->k_codes, pl->io_scratch, n, fi.code_field, Cm[fi.code_field], pl->status, st);
+        break;
+    case SCOPE_CLUSTER_SIZES: launch_check_range_i32(pl->n_c, n, 0, p.N, pl->status, st); break;
+    case SCOPE_TOPP_COUNT: launch_check_range_i32(pl->t_c, n, 1, p.N, pl->status, st); break;
+    case SCOPE_BASE_COUNT: launch_check_range_i32(pl->b_c, n, 1, p.N, pl->status, st); break;
+    case SCOPE_K_HEAD: launch_check_range_i32(pl->k_head, n, 1, p.N, pl->status, st); break;
+    case SCOPE_FINAL_COUNT: launch_check_range_i32(pl->r_c, n, 1, p.N, pl->status, st); break;
+    case SCOPE_KEY_OFFSETS: launch_check_offsets_i64(pl->key_offsets, n, p.index_capacity, pl->status, st); break;
+    case SCOPE_KEY_INDICES: launch_check_range_i32(pl->key_indices, n, 0, p.N - 1, pl->status, st); break;
+    case SCOPE_Q_PERM: launch_check_range_i32(pl->q_perm, n, 0, p.N - 1, pl->status, st); break;
+    case SCOPE_Q_OFFSETS:
+        launch_check_offsets_i32(pl->q_offsets, pl->BH, p.Cq + 1, p.N, pl->status, st);
+        {   // row tiles of the attention kernel follow from the offsets
+            GroupArgs a{};
+            a.BH = pl->BH; a.N = p.N; a.Cq = p.Cq;
+            a.q_offsets = pl->q_offsets; a.tile_offsets = pl->tile_offsets; a.tile_rows = kAttnTileRows;
+            launch_tiles_from_offsets(a, st);
+        }
+        break;
+    default: break;
+    }
+    return scope_plan_status(pl, stream, nullptr);
+}
+
+const char *scope_status_string(scope_status s)
+{
+    switch (s) {
+    case SCOPE_OK: return "ok";
+    case SCOPE_ERR_INVALID_ARG: return "invalid argument";
+    case SCOPE_ERR_UNSUPPORTED: return "unsupported configuration";
+    case SCOPE_ERR_ALIGNMENT: return "pointer or stride not 16-byte aligned";
+    case SCOPE_ERR_WORKSPACE: return "workspace too small";
+    case SCOPE_ERR_CAPACITY: return "key-index capacity too small";
+    case SCOPE_ERR_BAD_PLAN: return "inconsistent plan arrays";
+    case SCOPE_ERR_TIMEOUT: return "device-side wait timed out";
+    case SCOPE_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+int64_t scope_kfix_from_alpha(int64_t N, int64_t num, int64_t den)
+{
+    if (N < 1 || num < 1 || den < 1 || num > den || N > (int64_t)1 << 40 || num > (int64_t)1 << 20)
+        return -1;
+    return (N * num + den - 1) / den;
+}
+
+int64_t scope_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

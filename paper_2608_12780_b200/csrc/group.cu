@@ -1,0 +1,132 @@
+// Query grouping: tokens of one head ordered by query cluster (the index sets Q_c of Algorithm 1
+// lines 2-4 written as a permutation), ascending token index inside a cluster, plus the offsets
+// of every cluster and of its row tiles for the attention kernel.
+#include "scope_internal.cuh"
+
+namespace scope {
+
+namespace {
+
+// one block per head: offsets from the cluster sizes
+__global__ void __launch_bounds__(1024) group_offsets_kernel(GroupArgs a)
+{
+    __shared__ int wq[32], wt[32];
+    __shared__ int carry_q, carry_t;
+    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0)
+        carry_q = carry_t = 0;
+    __syncthreads();
+    for (int base = 0; base < a.Cq; base += blockDim.x) {
+        const int c = base + tid;
+        const int n = c < a.Cq ? a.n_c[(size_t)bh * a.Cq + c] : 0;
+        const int t = (n + a.tile_rows - 1) / a.tile_rows;
+        int iq = n, it = t;
+        for (int o = 1; o < 32; o <<= 1) {
+            int uq = __shfl_up_sync(0xffffffffu, iq, o), ut = __shfl_up_sync(0xffffffffu, it, o);
+            if (lane >= o) {
+                iq += uq;
+                it += ut;
+            }
+        }
+        if (lane == 31) {
+            wq[warp] = iq;
+            wt[warp] = it;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            int vq = wq[lane], vt = wt[lane];
+            int sq = vq, stt = vt;
+            for (int o = 1; o < 32; o <<= 1) {
+                int uq = __shfl_up_sync(0xffffffffu, sq, o), ut = __shfl_up_sync(0xffffffffu, stt, o);
+                if (lane >= o) {
+                    sq += uq;
+                    stt += ut;
+                }
+            }
+            wq[lane] = sq - vq;
+            wt[lane] = stt - vt;
+        }
+        __syncthreads();
+        const int eq = carry_q + wq[warp] + iq - n, et = carry_t + wt[warp] + it - t;
+        if (c < a.Cq) {
+            a.q_offsets[(size_t)bh * (a.Cq + 1) + c] = eq;
+            a.tile_offsets[(size_t)bh * (a.Cq + 1) + c] = et;
+        }
+        __syncthreads();
+        if (tid == blockDim.x - 1) {
+            carry_q = eq + n;
+            carry_t = et + t;
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        a.q_offsets[(size_t)bh * (a.Cq + 1) + a.Cq] = carry_q;
+        a.tile_offsets[(size_t)bh * (a.Cq + 1) + a.Cq] = carry_t;
+    }
+}
+
+// one warp per (head, cluster): stable compaction of the tokens labelled c
+__global__ void __launch_bounds__(256) group_scatter_kernel(GroupArgs a)
+{
+    const int bh = blockIdx.y, lane = threadIdx.x & 31;
+    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (c >= a.Cq)
+        return;
+    const int32_t *g = a.g + (size_t)bh * a.N;
+    int32_t *perm = a.q_perm + (size_t)bh * a.N;
+    int pos = a.q_offsets[(size_t)bh * (a.Cq + 1) + c];
+    const int end = a.q_offsets[(size_t)bh * (a.Cq + 1) + c + 1];
+    for (int j0 = 0; j0 < a.N; j0 += 128) {
+        int lab[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            int j = j0 + u * 32 + lane;
+            lab[u] = j < a.N ? __ldg(g + j) : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            uint32_t m = __ballot_sync(0xffffffffu, lab[u] == c);
+            if (lab[u] == c) {
+                int p = pos + __popc(m & ((1u << lane) - 1u));
+                if (p < end)  // holds whenever the sizes match the labels
+                    perm[p] = j0 + u * 32 + lane;
+            }
+            pos += __popc(m);
+        }
+    }
+}
+
+// row-tile offsets from cluster offsets alone (imported plans)
+__global__ void tiles_from_offsets_kernel(GroupArgs a)
+{
+    const int bh = blockIdx.x * blockDim.x + threadIdx.x;
+    if (bh >= a.BH)
+        return;
+    const int32_t *qo = a.q_offsets + (size_t)bh * (a.Cq + 1);
+    int32_t *to = a.tile_offsets + (size_t)bh * (a.Cq + 1);
+    int acc = 0;
+    for (int c = 0; c < a.Cq; ++c) {
+        to[c] = acc;
+        int n = qo[c + 1] - qo[c];
+        acc += n > 0 ? (n + a.tile_rows - 1) / a.tile_rows : 0;
+    }
+    to[a.Cq] = acc;
+}
+
+}  // namespace
+
+void launch_tiles_from_offsets(const GroupArgs &a, cudaStream_t st)
+{
+    tiles_from_offsets_kernel<<<(a.BH + 63) / 64, 64, 0, st>>>(a);
+    count_launch();
+}
+
+void launch_group(const GroupArgs &a, cudaStream_t st)
+{
+    group_offsets_kernel<<<a.BH, 1024, 0, st>>>(a);
+    dim3 grid((a.Cq + 7) / 8, a.BH);
+    group_scatter_kernel<<<grid, 256, 0, st>>>(a);
+    count_launch(2);
+}
+
+}  // namespace scope

@@ -1,0 +1,361 @@
+// K-means of Algorithm 1 line 1 (queries, all channels) and Algorithm 2 line 3 (keys, one
+// clustering per RoPE channel range): nearest centroid as in Eq. 3, member mean as in Eq. 2.
+//
+// One Lloyd iteration = kmeans_assign_kernel (labels + member sums in one read of X)
+// followed by kmeans_finalize_kernel (means, squared norms).
+//
+// Labels are decided in fp64: a fast fp32 pass computes |u|^2 - 2 x.u for every
+// (token, centroid) pair and keeps the two smallest values per token; whenever their gap is
+// inside the worst-case rounding error of that pass, the token is re-evaluated with the
+// plain sum of squared differences in fp64, channel by channel, lowest index winning a
+// tie.  Member sums are accumulated in fp64 (sums of bf16 values are exact there, so their
+// order does not matter) and rounded once to fp32 after the division.
+#include "scope_internal.cuh"
+
+namespace scope {
+
+namespace {
+
+constexpr int TM = 128;   // tokens per block
+constexpr int TC = 128;   // centroids per pass
+constexpr int KC = 16;    // channels per staged chunk
+constexpr int NT = 256;   // threads per block
+constexpr int MAX_FLAGGED = 3 * TM;
+
+__device__ __forceinline__ void merge2(float &best, float &second, int &arg, float ob, float os, int oa)
+{
+    float nsec = fminf(fmaxf(best, ob), fminf(second, os));
+    if (ob < best || (ob == best && oa < arg)) {
+        best = ob;
+        arg = oa;
+    }
+    second = nsec;
+}
+
+__global__ void __launch_bounds__(NT) kmeans_assign_kernel(KmArgs a)
+{
+    __shared__ __align__(16) float xs[KC][TM + 4];
+    __shared__ __align__(16) float us[KC][TC + 4];
+    __shared__ float x2s[2][TM];
+    __shared__ int asg[3][TM];
+    __shared__ uint32_t sorted[3][TM];
+    __shared__ int flagged[MAX_FLAGGED];
+    __shared__ int nflagged;
+
+    const int tid = threadIdx.x;
+    const int bh = blockIdx.y;
+    const int b = bh / a.H, h = bh % a.H;
+    const bf16 *Xh = a.X + (int64_t)b * a.sb + (int64_t)h * a.sh;
+    const int tok0 = blockIdx.x * TM;
+    const int ty = tid >> 4, tx = tid & 15;
+
+    if (tid == 0)
+        nflagged = 0;
+    __syncthreads();
+
+    // staging roles: one token row and 8 consecutive channels per thread
+    const int ltok = tid & (TM - 1), koff = (tid >> 7) * 8;
+    const bool tok_ok = tok0 + ltok < a.N;
+    const bf16 *xrow = Xh + (int64_t)(tok0 + ltok) * a.sn;
+
+    for (int s = 0; s < a.nspaces; ++s) {
+        const KmSpace sp = a.sp[s];
+        const float *cent = sp.cent + (size_t)bh * sp.C * sp.D;
+        const float *unorm = sp.unorm + (size_t)bh * sp.C;
+        const int cbeg = sp.ch0 & ~(KC - 1);
+        const int cend = sp.ch0 + sp.D;
+        float best[8], second[8];
+        int arg[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            best[i] = INFINITY;
+            second[i] = INFINITY;
+            arg[i] = 0;
+        }
+        float x2 = 0.f;
+
+        for (int c0 = 0; c0 < sp.C; c0 += TC) {
+            float acc[8][8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    acc[i][j] = 0.f;
+
+            for (int k0 = cbeg; k0 < cend; k0 += KC) {
+                // stage X chunk (absolute channels k0..k0+15, zero outside the range / past N)
+                {
+                    float v[8];
+                    if (tok_ok) {
+                        uint4 raw = *reinterpret_cast<const uint4 *>(xrow + k0 + koff);
+                        const bf16 *e = reinterpret_cast<const bf16 *>(&raw);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            int ch = k0 + koff + q;
+                            v[q] = (ch >= sp.ch0 && ch < cend) ? __bfloat162float(e[q]) : 0.f;
+                        }
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            v[q] = 0.f;
+                    }
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        xs[koff + q][ltok] = v[q];
+                        if (c0 == 0)
+                            x2 = fmaf(v[q], v[q], x2);
+                    }
+                }
+                // stage centroid chunk
+                {
+                    int c = c0 + ltok;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        int ch = k0 + koff + q;
+                        float u = 0.f;
+                        if (c < sp.C && ch >= sp.ch0 && ch < cend)
+                            u = cent[(size_t)c * sp.D + (ch - sp.ch0)];
+                        us[koff + q][ltok] = u;
+                    }
+                }
+                __syncthreads();
+#pragma unroll
+                for (int k = 0; k < KC; ++k) {
+                    float4 xa = *reinterpret_cast<const float4 *>(&xs[k][ty * 8]);
+                    float4 xb = *reinterpret_cast<const float4 *>(&xs[k][ty * 8 + 4]);
+                    float4 ua = *reinterpret_cast<const float4 *>(&us[k][tx * 8]);
+                    float4 ub = *reinterpret_cast<const float4 *>(&us[k][tx * 8 + 4]);
+                    float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+                    float uv[8] = {ua.x, ua.y, ua.z, ua.w, ub.x, ub.y, ub.z, ub.w};
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            acc[i][j] = fmaf(xv[i], uv[j], acc[i][j]);
+                }
+                __syncthreads();
+            }
+            // |u|^2 - 2 x.u, running two smallest per token
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                int c = c0 + tx * 8 + j;
+                float un = c < sp.C ? __ldg(unorm + c) : INFINITY;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float dist = c < sp.C ? fmaf(-2.f, acc[i][j], un) : INFINITY;
+                    if (dist < best[i]) {
+                        second[i] = best[i];
+                        best[i] = dist;
+                        arg[i] = c;
+                    } else if (dist < second[i]) {
+                        second[i] = dist;
+                    }
+                }
+            }
+        }
+        // squared norm of the token's slice: two staging threads per token
+        x2s[tid >> 7][ltok] = x2;
+        // merge across the 16 threads that share a token row
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+#pragma unroll
+            for (int m = 8; m >= 1; m >>= 1) {
+                float ob = __shfl_xor_sync(0xffffffffu, best[i], m);
+                float os = __shfl_xor_sync(0xffffffffu, second[i], m);
+                int oa = __shfl_xor_sync(0xffffffffu, arg[i], m);
+                merge2(best[i], second[i], arg[i], ob, os, oa);
+            }
+        }
+        __syncthreads();  // x2s visible
+        if (tx == 0) {
+            const float u2max = __ldg(sp.u2max + bh);
+            const int span = ((cend + KC - 1) & ~(KC - 1)) - cbeg;
+            // worst-case error of two fp32 evaluations of |u|^2 - 2 x.u with `span` terms
+            const float kappa = 4.f * (float)(span + 8) * 5.9604645e-8f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                int lt = ty * 8 + i;
+                asg[s][lt] = arg[i];
+                float tol = kappa * (u2max + x2s[0][lt] + x2s[1][lt]);
+                if (tok0 + lt < a.N && second[i] - best[i] <= tol) {
+                    int slot = atomicAdd(&nflagged, 1);
+                    flagged[slot] = (s << 16) | lt;
+                }
+            }
+        }
+        __syncthreads();
+    }
+
+    // fp64 re-evaluation of the close calls: one warp per token, centroids spread over lanes
+    {
+        const int warp = tid >> 5, lane = tid & 31;
+        const int nf = nflagged;
+        for (int f = warp; f < nf; f += NT / 32) {
+            const int s = flagged[f] >> 16, lt = flagged[f] & 0xffff;
+            const KmSpace sp = a.sp[s];
+            const float *cent = sp.cent + (size_t)bh * sp.C * sp.D;
+            const bf16 *x = Xh + (int64_t)(tok0 + lt) * a.sn + sp.ch0;
+            double bd = INFINITY;
+            int ba = 0x7fffffff;
+            for (int c = lane; c < sp.C; c += 32) {
+                const float *u = cent + (size_t)c * sp.D;
+                double dist = 0.0;
+                for (int ch = 0; ch < sp.D; ++ch) {
+                    double diff = __dsub_rn((double)__bfloat162float(x[ch]), (double)u[ch]);
+                    dist = __dadd_rn(dist, __dmul_rn(diff, diff));
+                }
+                if (dist < bd) {
+                    bd = dist;
+                    ba = c;
+                }
+            }
+#pragma unroll
+            for (int m = 16; m >= 1; m >>= 1) {
+                double od = __shfl_xor_sync(0xffffffffu, bd, m);
+                int oa = __shfl_xor_sync(0xffffffffu, ba, m);
+                if (od < bd || (od == bd && oa < ba)) {
+                    bd = od;
+                    ba = oa;
+                }
+            }
+            if (lane == 0)
+                asg[s][lt] = ba;
+        }
+    }
+    __syncthreads();
+
+    // labels out
+    if (tid < TM && tok0 + tid < a.N) {
+        if (a.nspaces == 1)
+            a.assign[(size_t)bh * a.N + tok0 + tid] = asg[0][tid];
+        else
+            a.codes[(size_t)bh * a.N + tok0 + tid] =
+                (uint32_t)asg[0][tid] | ((uint32_t)asg[1][tid] << kCodeBits) | ((uint32_t)asg[2][tid] << (2 * kCodeBits));
+    }
+
+    // order the tile's tokens by label (rank by counting), then add each run of equal labels once
+    for (int e = tid; e < a.nspaces * TM; e += NT) {
+        int s = e / TM, lt = e % TM;
+        uint32_t key = (tok0 + lt < a.N ? (uint32_t)asg[s][lt] : (uint32_t)kMaxClusters) << 8 | (uint32_t)lt;
+        int rank = 0;
+        for (int o = 0; o < TM; ++o) {
+            uint32_t ok = (tok0 + o < a.N ? (uint32_t)asg[s][o] : (uint32_t)kMaxClusters) << 8 | (uint32_t)o;
+            rank += ok < key;
+        }
+        sorted[s][rank] = key;
+    }
+    __syncthreads();
+    {
+        const int ch = tid & (kHeadDim - 1), half = tid >> 7;
+        int s = 0;
+        while (s + 1 < a.nspaces && ch >= a.sp[s].ch0 + a.sp[s].D)
+            ++s;
+        const KmSpace sp = a.sp[s];
+        if (ch >= sp.ch0 && ch < sp.ch0 + sp.D) {
+            const int rel = ch - sp.ch0;
+            double *sums = sp.sums + (size_t)bh * sp.C * sp.D;
+            int32_t *counts = sp.counts + (size_t)bh * sp.C;
+            int cur = -1, run = 0;
+            double acc = 0.0;
+            for (int l = half * (TM / 2); l < (half + 1) * (TM / 2); ++l) {
+                uint32_t key = sorted[s][l];
+                int cl = (int)(key >> 8), lt = (int)(key & 255u);
+                if (cl >= kMaxClusters)
+                    break;
+                if (cl != cur) {
+                    if (cur >= 0) {
+                        atomicAdd(sums + (size_t)cur * sp.D + rel, acc);
+                        if (rel == 0)
+                            atomicAdd(counts + cur, run);
+                    }
+                    cur = cl;
+                    acc = 0.0;
+                    run = 0;
+                }
+                acc += (double)__bfloat162float(Xh[(int64_t)(tok0 + lt) * a.sn + ch]);
+                ++run;
+            }
+            if (cur >= 0) {
+                atomicAdd(sums + (size_t)cur * sp.D + rel, acc);
+                if (rel == 0)
+                    atomicAdd(counts + cur, run);
+            }
+        }
+    }
+}
+
+// mode 0: centroids from member sums (empty clusters keep theirs); mode 1: evenly strided tokens;
+// mode 2: centroids as they are (imported).  All refresh the squared norms and clear the sums for
+// the next iteration.
+__global__ void __launch_bounds__(256) kmeans_finalize_kernel(KmArgs a, int mode)
+{
+    __shared__ float red[256];
+    const int bh = blockIdx.x, s = blockIdx.y;
+    const KmSpace sp = a.sp[s];
+    const int b = bh / a.H, h = bh % a.H;
+    const bf16 *Xh = a.X + (int64_t)b * a.sb + (int64_t)h * a.sh;
+    float *cent = sp.cent + (size_t)bh * sp.C * sp.D;
+    double *sums = sp.sums + (size_t)bh * sp.C * sp.D;
+    int32_t *counts = sp.counts + (size_t)bh * sp.C;
+
+    for (int e = threadIdx.x; e < sp.C * sp.D; e += blockDim.x) {
+        int r = e / sp.D, ch = e % sp.D;
+        if (mode == 1) {
+            int64_t tok = ((int64_t)r * a.N) / sp.C;
+            cent[e] = __bfloat162float(Xh[tok * a.sn + sp.ch0 + ch]);
+        } else if (mode == 0) {
+            int n = counts[r];
+            if (n > 0)
+                cent[e] = (float)(sums[e] / (double)n);
+        }
+        sums[e] = 0.0;
+    }
+    __syncthreads();
+    float mx = 0.f;
+    for (int r = threadIdx.x; r < sp.C; r += blockDim.x) {
+        float n2 = 0.f;
+        for (int ch = 0; ch < sp.D; ++ch)
+            n2 = fmaf(cent[(size_t)r * sp.D + ch], cent[(size_t)r * sp.D + ch], n2);
+        sp.unorm[(size_t)bh * sp.C + r] = n2;
+        mx = fmaxf(mx, n2);
+        if (mode == 0 && sp.sizes)
+            sp.sizes[(size_t)bh * sp.C + r] = counts[r];
+        counts[r] = 0;
+    }
+    red[threadIdx.x] = mx;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o)
+            red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + o]);
+        __syncthreads();
+    }
+    if (threadIdx.x == 0)
+        sp.u2max[bh] = red[0];
+}
+
+}  // namespace
+
+void launch_kmeans_init(const KmArgs &a, cudaStream_t st)
+{
+    dim3 grid(a.B * a.H, a.nspaces);
+    kmeans_finalize_kernel<<<grid, 256, 0, st>>>(a, 1);
+    count_launch();
+}
+
+void launch_kmeans_norms(const KmArgs &a, cudaStream_t st)
+{
+    dim3 grid(a.B * a.H, a.nspaces);
+    kmeans_finalize_kernel<<<grid, 256, 0, st>>>(a, 2);
+    count_launch();
+}
+
+void launch_kmeans_iteration(const KmArgs &a, cudaStream_t st)
+{
+    dim3 grid((a.N + TM - 1) / TM, a.B * a.H);
+    kmeans_assign_kernel<<<grid, NT, 0, st>>>(a);
+    dim3 fgrid(a.B * a.H, a.nspaces);
+    kmeans_finalize_kernel<<<fgrid, 256, 0, st>>>(a, 0);
+    count_launch(2);
+}
+
+}  // namespace scope

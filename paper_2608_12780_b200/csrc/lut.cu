@@ -1,0 +1,57 @@
+// Score tables of Eq. 5 / Algorithm 2 line 4: P_m[c, r] = < qbar_c[I_m], u_r^m >.
+// A few MFLOP per head: one thread per entry, fp64 accumulation channel by channel,
+// one rounding to fp32 (products of two fp32 values are exact in fp64).
+#include "scope_internal.cuh"
+
+namespace scope {
+
+namespace {
+
+struct LutArgs {
+    int Cq, d;
+    const float *qcent;  // [BH, Cq, d]
+    int ch0[3], D[3], C[3];
+    const float *ucent[3];  // [BH, C_m, d_m]
+    float *lut[3];          // [BH, Cq, C_m]
+};
+
+__global__ void __launch_bounds__(256) lut_kernel(LutArgs a)
+{
+    const int bh = blockIdx.x, m = blockIdx.y;
+    const int C = a.C[m], D = a.D[m], ch0 = a.ch0[m];
+    const float *q = a.qcent + (size_t)bh * a.Cq * a.d + ch0;
+    const float *u = a.ucent[m] + (size_t)bh * C * D;
+    float *P = a.lut[m] + (size_t)bh * a.Cq * C;
+    for (int e = blockIdx.z * blockDim.x + threadIdx.x; e < a.Cq * C; e += gridDim.z * blockDim.x) {
+        int c = e / C, r = e % C;
+        double acc = 0.0;
+        for (int ch = 0; ch < D; ++ch)
+            acc = __dadd_rn(acc, __dmul_rn((double)q[(size_t)c * a.d + ch], (double)u[(size_t)r * D + ch]));
+        P[e] = (float)acc;
+    }
+}
+
+}  // namespace
+
+void launch_lut(int BH, int Cq, int d, const float *qcent, const KmSpace *ksp, float *const *lut, cudaStream_t st)
+{
+    LutArgs a;
+    a.Cq = Cq;
+    a.d = d;
+    a.qcent = qcent;
+    int maxC = 1;
+    for (int m = 0; m < 3; ++m) {
+        a.ch0[m] = ksp[m].ch0;
+        a.D[m] = ksp[m].D;
+        a.C[m] = ksp[m].C;
+        a.ucent[m] = ksp[m].cent;
+        a.lut[m] = lut[m];
+        maxC = ksp[m].C > maxC ? ksp[m].C : maxC;
+    }
+    int z = (Cq * maxC + 255) / 256;
+    z = z < 1 ? 1 : (z > 16 ? 16 : z);
+    lut_kernel<<<dim3(BH, 3, z), 256, 0, st>>>(a);
+    count_launch();
+}
+
+}  // namespace scope

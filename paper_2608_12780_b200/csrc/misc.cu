@@ -1,0 +1,107 @@
+// Small helper kernels of plan import / export: range checks that report through the status word
+// instead of letting a malformed array be dereferenced later, and (un)packing of the key codes.
+#include "scope_internal.cuh"
+
+namespace scope {
+
+namespace {
+
+__global__ void check_range_i32_kernel(const int32_t *x, int64_t n, int32_t lo, int32_t hi, int32_t *status)
+{
+    bool bad = false;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        bad |= x[i] < lo || x[i] > hi;
+    if (__syncthreads_or(bad) && threadIdx.x == 0)
+        atomicCAS(status + ST_CODE, 0, (int)SCOPE_ERR_BAD_PLAN);
+}
+
+__global__ void check_offsets_i64_kernel(const int64_t *x, int64_t n, int64_t cap, int32_t *status)
+{
+    bool bad = false;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        bad |= x[i] < 0 || x[i] > cap;
+        if (i == 0)
+            bad |= x[0] != 0;
+        else
+            bad |= x[i] < x[i - 1];
+    }
+    if (__syncthreads_or(bad) && threadIdx.x == 0)
+        atomicCAS(status + ST_CODE, 0, (int)SCOPE_ERR_BAD_PLAN);
+}
+
+__global__ void check_offsets_i32_kernel(const int32_t *x, int rows, int cols, int32_t last, int32_t *status)
+{
+    bool bad = false;
+    const int64_t n = (int64_t)rows * cols;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        int c = (int)(i % cols);
+        bad |= x[i] < 0 || x[i] > last;
+        if (c == 0)
+            bad |= x[i] != 0;
+        else
+            bad |= x[i] < x[i - 1];
+        if (c == cols - 1)
+            bad |= x[i] != last;
+    }
+    if (__syncthreads_or(bad) && threadIdx.x == 0)
+        atomicCAS(status + ST_CODE, 0, (int)SCOPE_ERR_BAD_PLAN);
+}
+
+__global__ void pack_codes_kernel(uint32_t *codes, const int32_t *src, int64_t n, int field, int C, int32_t *status)
+{
+    bool bad = false;
+    const int sh = field * kCodeBits;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        int v = src[i];
+        if (v < 0 || v >= C) {
+            bad = true;
+            v = 0;
+        }
+        codes[i] = (codes[i] & ~(kCodeMask << sh)) | ((uint32_t)v << sh);
+    }
+    if (__syncthreads_or(bad) && threadIdx.x == 0)
+        atomicCAS(status + ST_CODE, 0, (int)SCOPE_ERR_BAD_PLAN);
+}
+
+__global__ void unpack_codes_kernel(const uint32_t *codes, int32_t *dst, int64_t n, int field)
+{
+    const int sh = field * kCodeBits;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        dst[i] = (int32_t)((codes[i] >> sh) & kCodeMask);
+}
+
+int blocks_for(int64_t n)
+{
+    int64_t b = (n + 255) / 256;
+    return (int)(b < 1 ? 1 : (b > 2048 ? 2048 : b));
+}
+
+}  // namespace
+
+void launch_check_range_i32(const int32_t *x, int64_t n, int32_t lo, int32_t hi, int32_t *status, cudaStream_t st)
+{
+    check_range_i32_kernel<<<blocks_for(n), 256, 0, st>>>(x, n, lo, hi, status);
+    count_launch();
+}
+void launch_check_offsets_i64(const int64_t *x, int64_t n, int64_t cap, int32_t *status, cudaStream_t st)
+{
+    check_offsets_i64_kernel<<<blocks_for(n), 256, 0, st>>>(x, n, cap, status);
+    count_launch();
+}
+void launch_check_offsets_i32(const int32_t *x, int rows, int cols, int32_t last, int32_t *status, cudaStream_t st)
+{
+    check_offsets_i32_kernel<<<blocks_for((int64_t)rows * cols), 256, 0, st>>>(x, rows, cols, last, status);
+    count_launch();
+}
+void launch_pack_codes(uint32_t *codes, const int32_t *src, int64_t n, int field, int C, int32_t *status, cudaStream_t st)
+{
+    pack_codes_kernel<<<blocks_for(n), 256, 0, st>>>(codes, src, n, field, C, status);
+    count_launch();
+}
+void launch_unpack_codes(const uint32_t *codes, int32_t *dst, int64_t n, int field, cudaStream_t st)
+{
+    unpack_codes_kernel<<<blocks_for(n), 256, 0, st>>>(codes, dst, n, field);
+    count_launch();
+}
+
+}  // namespace scope

@@ -1,0 +1,111 @@
+// Internal declarations shared by the kernels of the SCOPE library (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "scope.h"
+
+namespace scope {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kHeadDim = 128;
+constexpr int kMaxClusters = 1024;  // codes are packed in 10-bit fields
+constexpr int kCodeBits = 10;
+constexpr uint32_t kCodeMask = (1u << kCodeBits) - 1u;
+
+// device status words at the start of the workspace
+enum { ST_CODE = 0, ST_NEEDED_LO = 2 /* int64 at [2..3] */, ST_WORDS = 64 };
+
+// One clustered channel range: the whole head dimension for queries, one RoPE range for keys.
+struct KmSpace {
+    int ch0, D, C;
+    float *cent;      // [BH, C, D]
+    float *unorm;     // [BH, C]     squared norms of the centroids (fp32)
+    float *u2max;     // [BH]        largest squared centroid norm
+    double *sums;     // [BH, C, D]  member sums of the running iteration
+    int32_t *counts;  // [BH, C]
+    int32_t *sizes;   // [BH, C] or null: copy of the member counts of the last assignment
+};
+
+struct KmArgs {
+    const bf16 *X;
+    int64_t sb, sh, sn;
+    int B, H, N;
+    int nspaces;       // 1 (queries) or 3 (keys)
+    KmSpace sp[3];
+    int32_t *assign;   // [BH, N] labels (nspaces == 1)
+    uint32_t *codes;   // [BH, N] packed labels (nspaces == 3)
+};
+
+// Per (head, query cluster) result of the selection stage that later kernels read.
+struct RowState {
+    uint32_t tau_key;   // order-preserving key of the threshold logit of the Top-p prefix
+    int32_t cnt_above;  // keys strictly above it
+};
+
+struct SelectArgs {
+    int BH, N, Cq, Ct, Ch, Cw;
+    float scale;
+    float top_p;
+    int k_fix;
+    int64_t capacity;
+    const uint32_t *codes;   // [BH, N]
+    const float *lutT, *lutH, *lutW;  // [BH, Cq, Cm]
+    const int32_t *n_c;      // [BH, Cq]
+    int32_t *t_c, *b_c, *r_c, *k_head;
+    RowState *rows;          // [BH, Cq]
+    int64_t *key_offsets;    // [BH*Cq + 1]
+    int32_t *key_indices;
+    int32_t *status;
+};
+
+struct GroupArgs {
+    int BH, N, Cq;
+    const int32_t *g;        // [BH, N]
+    const int32_t *n_c;      // [BH, Cq]
+    int32_t *q_perm;         // [BH, N]
+    int32_t *q_offsets;      // [BH, Cq + 1]
+    int32_t *tile_offsets;   // [BH, Cq + 1] prefix of ceil(n_c / tile rows)
+    int tile_rows;
+};
+
+struct AttnArgs {
+    const bf16 *Q, *K, *V;
+    bf16 *O;
+    int64_t sb, sh, sn;
+    int B, H, N, Cq;
+    float scale;
+    int dense;               // 1: every key, identity grouping (Eq. 1)
+    const int32_t *q_perm, *q_offsets, *tile_offsets;
+    const int32_t *r_c;
+    const int64_t *key_offsets;
+    const int32_t *key_indices;
+    const int32_t *status;   // kernels skip all work unless status[ST_CODE] == 0
+    int max_tiles_per_head;
+};
+
+// launchers (each enqueues on `st` and bumps the launch counter)
+void launch_kmeans_init(const KmArgs &a, cudaStream_t st);
+void launch_kmeans_norms(const KmArgs &a, cudaStream_t st);
+void launch_kmeans_iteration(const KmArgs &a, cudaStream_t st);
+void launch_lut(int BH, int Cq, int d, const float *qcent, const KmSpace *ksp /*3*/, float *const *lut,
+                cudaStream_t st);
+void launch_select(const SelectArgs &a, cudaStream_t st);
+void launch_group(const GroupArgs &a, cudaStream_t st);
+void launch_tiles_from_offsets(const GroupArgs &a, cudaStream_t st);
+void launch_attn(const AttnArgs &a, cudaStream_t st);
+constexpr int kAttnTileRows = 64;
+
+void count_launch(int n = 1);
+
+// validation kernels used by scope_plan_import
+void launch_check_range_i32(const int32_t *x, int64_t n, int32_t lo, int32_t hi, int32_t *status, cudaStream_t st);
+void launch_check_offsets_i64(const int64_t *x, int64_t n, int64_t cap, int32_t *status, cudaStream_t st);
+void launch_check_offsets_i32(const int32_t *x, int rows, int cols, int32_t last, int32_t *status, cudaStream_t st);
+void launch_pack_codes(uint32_t *codes, const int32_t *src, int64_t n, int field, int C, int32_t *status, cudaStream_t st);
+void launch_unpack_codes(const uint32_t *codes, int32_t *dst, int64_t n, int field, cudaStream_t st);
+
+}  // namespace scope

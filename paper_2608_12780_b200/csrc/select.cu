@@ -1,0 +1,585 @@
+// Selection stage: Eq. 6 (proxy logits as three table reads), Eq. 7 (Top-p count), Eq. 8 (floor),
+// Eq. 9 (per-head k), Eq. 10 (final counts and key sets) — Algorithm 3.
+//
+// No row of the proxy-logit matrix is ever stored or sorted.  A logit is recomputed from the
+// key's packed code whenever it is needed, mapped to an order-preserving 32-bit key, and the
+// two order statistics the method needs are found by a three-level radix descent (11+11+10
+// bits) over histograms held in shared memory:
+//   * Top-p: histograms carry the member count and the softmax mass (fp64) of every bin; the
+//     descent follows the bin in which the cumulative mass, taken from the largest logit down,
+//     reaches rho * Z.  Keys with equal logits are consecutive in the ranking, so inside the
+//     final group the count is closed-form.
+//   * rank r_c: the same descent on counts alone, only for clusters whose r_c differs from t_c.
+// The key set is then written by one ordered pass over the keys: everything above the
+// threshold logit, plus the lowest-indexed keys of the threshold group (equal logits are
+// ranked by ascending key index), in ascending key index.
+#include "scope_internal.cuh"
+
+namespace scope {
+
+namespace {
+
+constexpr int R = 4;          // query clusters (rows) per block: they share every code read
+constexpr int NT = 512;       // threads per block
+constexpr int NWARP = NT / 32;
+constexpr int NB = 2048;      // bins per level
+constexpr int LEVELS = 3;
+__device__ __constant__ int kShift[LEVELS] = {21, 10, 0};
+__device__ __constant__ int kBits[LEVELS] = {11, 11, 10};
+
+__device__ __forceinline__ uint32_t order_key(float raw)
+{
+    uint32_t u = __float_as_uint(raw + 0.0f);  // -0 -> +0
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_value(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+struct RowTables {
+    const float *T, *H, *W;  // shared-memory rows of the three tables
+};
+
+__device__ __forceinline__ float proxy_raw(const RowTables &t, uint32_t code)
+{
+    // Eq. 6 before the 1/sqrt(d) factor, in this order
+    float a = t.T[code & kCodeMask] + t.H[(code >> kCodeBits) & kCodeMask];
+    return a + t.W[code >> (2 * kCodeBits)];
+}
+
+__device__ __forceinline__ void load_tables(const SelectArgs &a, int bh, int c0, float *lut, RowTables *rt)
+{
+    const int CS = a.Ct + a.Ch + a.Cw;
+    for (int e = threadIdx.x; e < R * CS; e += NT) {
+        int r = e / CS, o = e % CS;
+        int c = min(c0 + r, a.Cq - 1);
+        float v;
+        if (o < a.Ct)
+            v = a.lutT[((size_t)bh * a.Cq + c) * a.Ct + o];
+        else if (o < a.Ct + a.Ch)
+            v = a.lutH[((size_t)bh * a.Cq + c) * a.Ch + (o - a.Ct)];
+        else
+            v = a.lutW[((size_t)bh * a.Cq + c) * a.Cw + (o - a.Ct - a.Ch)];
+        lut[e] = v;
+    }
+    for (int r = 0; r < R; ++r) {
+        rt[r].T = lut + r * CS;
+        rt[r].H = rt[r].T + a.Ct;
+        rt[r].W = rt[r].H + a.Ch;
+    }
+}
+
+// Descending walk over one row's bins by one warp: finds the first bin (from the top) at which
+// carried + cumulative weight reaches `target`.  W is uint32 counts (uint64 sums) or fp64 masses.
+// Returns the bin (or -1), and the cumulative weight and count strictly above it.
+template <typename W, typename ACC>
+__device__ __forceinline__ int descend(const W *w, const uint32_t *cnt, int nb, ACC carried, ACC target,
+                                       ACC &w_above, int64_t &c_above, int &last_nonempty)
+{
+    const int lane = threadIdx.x & 31;
+    const int per = nb / 32;
+    // lane l owns bins [nb-1 - l*per, nb - (l+1)*per], walked downwards
+    ACC lsum = 0;
+    int64_t lcnt = 0;
+    int llast = -1;
+    for (int i = 0; i < per; ++i) {
+        int bin = nb - 1 - (lane * per + i);
+        lsum += (ACC)w[bin];
+        uint32_t c = cnt[bin];
+        lcnt += c;
+        if (c)
+            llast = bin;
+    }
+    // exclusive prefix over lanes, in lane order
+    ACC pre = lsum;
+    int64_t cpre = lcnt;
+    for (int o = 1; o < 32; o <<= 1) {
+        ACC v = __shfl_up_sync(0xffffffffu, pre, o);
+        int64_t cv = __shfl_up_sync(0xffffffffu, cpre, o);
+        if (lane >= o) {
+            pre += v;
+            cpre += cv;
+        }
+    }
+    ACC excl = pre - lsum;  // exact for integers; for fp64 recomputed below
+    int64_t cexcl = cpre - lcnt;
+    if (sizeof(ACC) == sizeof(double)) {
+        // avoid the cancellation of pre - lsum: take the inclusive prefix of the previous lane
+        ACC up = __shfl_up_sync(0xffffffffu, pre, 1);
+        excl = lane == 0 ? (ACC)0 : up;
+    }
+    bool crosses = carried + pre >= target;  // inclusive prefix reaches the target
+    uint32_t ball = __ballot_sync(0xffffffffu, crosses);
+    // lowest non-empty bin of the whole row (fallback when rounding leaves no crossing)
+    int lowest = llast;
+    for (int o = 16; o > 0; o >>= 1) {
+        int v = __shfl_xor_sync(0xffffffffu, lowest, o);
+        lowest = (lowest < 0) ? v : (v < 0 ? lowest : min(lowest, v));
+    }
+    last_nonempty = lowest;
+    int found = -1;
+    ACC fa = 0;
+    int64_t fc = 0;
+    if (ball) {
+        int src = __ffs(ball) - 1;
+        if (lane == src) {
+            ACC run = carried + excl;
+            int64_t rc = cexcl;
+            for (int i = 0; i < per; ++i) {
+                int bin = nb - 1 - (lane * per + i);
+                ACC nxt = run + (ACC)w[bin];
+                if (cnt[bin] && nxt >= target) {
+                    found = bin;
+                    break;
+                }
+                run = nxt;
+                rc += cnt[bin];
+            }
+            if (found < 0) {  // inclusive prefix said yes, the walk rounded differently: take the lane's last bin
+                found = llast;
+                run = carried + excl;
+                rc = cexcl;
+                for (int i = 0; i < per; ++i) {
+                    int bin = nb - 1 - (lane * per + i);
+                    if (bin == found)
+                        break;
+                    run += (ACC)w[bin];
+                    rc += cnt[bin];
+                }
+            }
+            fa = run - carried;
+            fc = rc;
+        }
+        found = __shfl_sync(0xffffffffu, found, src);
+        fa = __shfl_sync(0xffffffffu, fa, src);
+        fc = __shfl_sync(0xffffffffu, fc, src);
+    }
+    w_above = fa;
+    c_above = fc;
+    return found;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Top-p count t_c (Eq. 7) for R query clusters of one head.
+__global__ void __launch_bounds__(NT, 2) select_topp_kernel(SelectArgs a)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *mass = reinterpret_cast<double *>(smem_raw);                   // [R][NB]
+    uint32_t *cnt = reinterpret_cast<uint32_t *>(mass + R * NB);           // [R][NB]
+    float *lut = reinterpret_cast<float *>(cnt + R * NB);
+    __shared__ uint32_t kmax[R];
+    __shared__ uint32_t prefix[R];
+    __shared__ double carried_mass[R];
+    __shared__ int64_t carried_cnt[R];
+    __shared__ double targetZ[R];
+
+    const int bh = blockIdx.y, c0 = blockIdx.x * R;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t *codes = a.codes + (size_t)bh * a.N;
+    RowTables lrt[R];
+    load_tables(a, bh, c0, lut, lrt);
+    if (tid < R) {
+        kmax[tid] = 0u;
+        prefix[tid] = 0u;
+        carried_mass[tid] = 0.0;
+        carried_cnt[tid] = 0;
+    }
+    __syncthreads();
+
+    // row maximum (softmax is evaluated with the maximum subtracted)
+    {
+        uint32_t m[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+            m[r] = 0u;
+        for (int j = tid; j < a.N; j += NT) {
+            uint32_t code = __ldg(codes + j);
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                m[r] = max(m[r], order_key(proxy_raw(lrt[r], code)));
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            uint32_t v = m[r];
+            for (int o = 16; o > 0; o >>= 1)
+                v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+            if (lane == 0)
+                atomicMax(&kmax[r], v);
+        }
+    }
+    __syncthreads();
+    double mx[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+        mx[r] = (double)__fmul_rn(key_value(kmax[r]), a.scale);
+
+    for (int lv = 0; lv < LEVELS; ++lv) {
+        const int shift = kShift[lv], nb = 1 << kBits[lv];
+        const int pshift = lv == 0 ? 32 : kShift[lv - 1];
+        for (int e = tid; e < R * NB; e += NT) {
+            cnt[e] = 0u;
+            mass[e] = 0.0;
+        }
+        __syncthreads();
+        uint32_t pf[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+            pf[r] = prefix[r];
+        for (int j = tid; j < a.N; j += NT) {
+            uint32_t code = __ldg(codes + j);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float raw = proxy_raw(lrt[r], code);
+                uint32_t key = order_key(raw);
+                if (lv == 0 || (key >> pshift) == pf[r]) {
+                    int bin = (key >> shift) & (nb - 1);
+                    double e = exp((double)__fmul_rn(raw + 0.0f, a.scale) - mx[r]);
+                    atomicAdd(&cnt[r * NB + bin], 1u);
+                    atomicAdd(&mass[r * NB + bin], e);
+                }
+            }
+        }
+        __syncthreads();
+        if (warp < R) {
+            const int r = warp;
+            const double *wm = mass + r * NB;
+            const uint32_t *wc = cnt + r * NB;
+            if (lv == 0) {
+                // Z: all bins, descending, fixed order
+                double z = 0.0;
+                for (int i = 0; i < NB / 32; ++i)
+                    z += wm[NB - 1 - (lane * (NB / 32) + i)];
+                for (int o = 16; o > 0; o >>= 1)
+                    z += __shfl_xor_sync(0xffffffffu, z, o);
+                if (lane == 0)
+                    targetZ[r] = (double)a.top_p * z;
+            }
+            __syncwarp();
+            double w_above;
+            int64_t c_above;
+            int lowest;
+            int bin = descend<double, double>(wm, wc, nb, carried_mass[r], targetZ[r], w_above, c_above, lowest);
+            if (bin < 0) {  // rounding left no crossing inside the followed bin: its last group closes it
+                bin = lowest;
+                w_above = 0.0;
+                c_above = 0;
+                if (lane == 0) {
+                    for (int b2 = nb - 1; b2 > bin; --b2) {
+                        w_above += wm[b2];
+                        c_above += wc[b2];
+                    }
+                }
+                w_above = __shfl_sync(0xffffffffu, w_above, 0);
+                c_above = __shfl_sync(0xffffffffu, c_above, 0);
+            }
+            if (lane == 0) {
+                carried_mass[r] += w_above;
+                carried_cnt[r] += c_above;
+                prefix[r] = (prefix[r] << kBits[lv]) | (uint32_t)bin;
+                if (lv == LEVELS - 1 && c0 + r < a.Cq) {
+                    // threshold group: m keys of equal logit e_tau each; smallest i with mass_above + i e >= target
+                    const uint32_t tau = prefix[r];
+                    const double m_tau = (double)wc[bin];
+                    const double e_tau = exp((double)__fmul_rn(key_value(tau), a.scale) - mx[r]);
+                    const double above = carried_mass[r], target = targetZ[r];
+                    double i = ceil((target - above) / e_tau);
+                    i = fmin(fmax(i, 1.0), m_tau);
+                    while (i > 1.0 && above + (i - 1.0) * e_tau >= target)
+                        i -= 1.0;
+                    while (i < m_tau && above + i * e_tau < target)
+                        i += 1.0;
+                    int64_t t = carried_cnt[r] + (int64_t)i;
+                    if (a.top_p >= 1.0f)
+                        t = a.N;
+                    const size_t row = (size_t)bh * a.Cq + c0 + r;
+                    a.t_c[row] = (int32_t)t;
+                    a.rows[row].tau_key = tau;
+                    a.rows[row].cnt_above = (int32_t)carried_cnt[r];
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Eq. 8, Eq. 9, Eq. 10 counts for every head, then the offsets of the key sets.
+__global__ void __launch_bounds__(1024) khead_kernel(SelectArgs a)
+{
+    __shared__ unsigned long long red[32];
+    __shared__ long long scan_carry, chunk_total;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int bh = 0; bh < a.BH; ++bh) {
+        unsigned long long num = 0;
+        for (int c = tid; c < a.Cq; c += blockDim.x) {
+            size_t row = (size_t)bh * a.Cq + c;
+            int b = max(a.t_c[row], a.k_fix);
+            a.b_c[row] = b;
+            num += (unsigned long long)a.n_c[row] * (unsigned long long)b;
+        }
+        for (int o = 16; o > 0; o >>= 1)
+            num += __shfl_xor_sync(0xffffffffu, num, o);
+        if (lane == 0)
+            red[warp] = num;
+        __syncthreads();
+        if (warp == 0) {
+            unsigned long long v = lane < (blockDim.x >> 5) ? red[lane] : 0ull;
+            for (int o = 16; o > 0; o >>= 1)
+                v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (lane == 0)
+                red[0] = v;
+        }
+        __syncthreads();
+        // sum of n_c over a head is N
+        const long long k = (long long)((red[0] + (unsigned long long)a.N - 1ull) / (unsigned long long)a.N);
+        if (tid == 0)
+            a.k_head[bh] = (int32_t)k;
+        for (int c = tid; c < a.Cq; c += blockDim.x) {
+            size_t row = (size_t)bh * a.Cq + c;
+            long long r = max((long long)a.b_c[row], k);
+            a.r_c[row] = (int32_t)min(r, (long long)a.N);
+        }
+        __syncthreads();
+    }
+    // exclusive scan of r_c over all (head, cluster) rows
+    if (tid == 0)
+        scan_carry = 0;
+    __syncthreads();
+    const int64_t rows = (int64_t)a.BH * a.Cq;
+    for (int64_t base = 0; base < rows; base += blockDim.x) {
+        const int64_t i = base + tid;
+        const long long v = i < rows ? a.r_c[i] : 0;
+        long long inc = v;
+        for (int o = 1; o < 32; o <<= 1) {
+            long long u = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o)
+                inc += u;
+        }
+        if (lane == 31)
+            red[warp] = (unsigned long long)inc;
+        __syncthreads();
+        if (warp == 0) {
+            const long long w = lane < (blockDim.x >> 5) ? (long long)red[lane] : 0;
+            long long winc = w;
+            for (int o = 1; o < 32; o <<= 1) {
+                long long u = __shfl_up_sync(0xffffffffu, winc, o);
+                if (lane >= o)
+                    winc += u;
+            }
+            red[lane] = (unsigned long long)(winc - w);
+            if (lane == 31)
+                chunk_total = winc;
+        }
+        __syncthreads();
+        if (i < rows)
+            a.key_offsets[i] = scan_carry + (long long)red[warp] + (inc - v);
+        __syncthreads();
+        if (tid == 0)
+            scan_carry += chunk_total;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        const long long total = scan_carry;
+        a.key_offsets[rows] = total;
+        *reinterpret_cast<long long *>(a.status + ST_NEEDED_LO) = total;
+        if (total > a.capacity && a.status[ST_CODE] == 0)
+            a.status[ST_CODE] = SCOPE_ERR_CAPACITY;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Key sets S_c (Eq. 10) for R query clusters of one head, ascending key index.
+__global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint32_t *cnt = reinterpret_cast<uint32_t *>(smem_raw);  // [R][NB]
+    float *lut = reinterpret_cast<float *>(cnt + R * NB);
+    __shared__ uint32_t tau[R];
+    __shared__ int need[R];       // threshold-group keys to take
+    __shared__ int todo[R];       // 1: rank descent still needed
+    __shared__ uint32_t prefix[R];
+    __shared__ int64_t carried[R];
+    __shared__ int wsel[R][NWARP], wtie[R][NWARP];
+    __shared__ int base_sel[R], base_tie[R];
+
+    if (a.status[ST_CODE] != 0)
+        return;  // e.g. index buffer too small: write nothing
+    const int bh = blockIdx.y, c0 = blockIdx.x * R;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t *codes = a.codes + (size_t)bh * a.N;
+    RowTables lrt[R];
+    load_tables(a, bh, c0, lut, lrt);
+    if (tid < R) {
+        const int c = c0 + tid;
+        int td = 0;
+        uint32_t t = 0u;
+        int nd = 0;
+        if (c < a.Cq) {
+            const size_t row = (size_t)bh * a.Cq + c;
+            const int r = a.r_c[row];
+            if (r >= a.N) {
+                t = 0u;          // every key is above key 0 or ties with it
+                nd = a.N;
+            } else if (r == a.t_c[row]) {
+                t = a.rows[row].tau_key;
+                nd = r - a.rows[row].cnt_above;
+            } else {
+                td = 1;
+            }
+        } else {
+            t = 0xffffffffu;     // padding row: selects nothing
+            nd = 0;
+        }
+        tau[tid] = t;
+        need[tid] = nd;
+        todo[tid] = td;
+        prefix[tid] = 0u;
+        carried[tid] = 0;
+        base_sel[tid] = 0;
+        base_tie[tid] = 0;
+    }
+    __syncthreads();
+    const bool any_todo = (todo[0] | todo[1] | todo[2] | todo[3]) != 0;
+    static_assert(R == 4, "any_todo spells out four rows");
+
+    if (any_todo) {
+        for (int lv = 0; lv < LEVELS; ++lv) {
+            const int shift = kShift[lv], nb = 1 << kBits[lv];
+            const int pshift = lv == 0 ? 32 : kShift[lv - 1];
+            for (int e = tid; e < R * NB; e += NT)
+                cnt[e] = 0u;
+            __syncthreads();
+            uint32_t pf[R];
+            int td[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                pf[r] = prefix[r];
+                td[r] = todo[r];
+            }
+            for (int j = tid; j < a.N; j += NT) {
+                uint32_t code = __ldg(codes + j);
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    if (!td[r])
+                        continue;
+                    uint32_t key = order_key(proxy_raw(lrt[r], code));
+                    if (lv == 0 || (key >> pshift) == pf[r])
+                        atomicAdd(&cnt[r * NB + ((key >> shift) & (nb - 1))], 1u);
+                }
+            }
+            __syncthreads();
+            if (warp < R && todo[warp]) {
+                const int r = warp;
+                const uint32_t *wc = cnt + r * NB;
+                const int64_t target = a.r_c[(size_t)bh * a.Cq + c0 + r];
+                int64_t w_above, c_above;
+                int lowest;
+                int bin = descend<uint32_t, int64_t>(wc, wc, nb, carried[r], target, w_above, c_above, lowest);
+                if (lane == 0) {
+                    carried[r] += c_above;
+                    prefix[r] = (prefix[r] << kBits[lv]) | (uint32_t)bin;
+                    if (lv == LEVELS - 1) {
+                        tau[r] = prefix[r];
+                        need[r] = (int)(target - carried[r]);
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+
+    // ordered emission
+    uint32_t tk[R];
+    int nd[R];
+    int64_t off[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        tk[r] = tau[r];
+        nd[r] = need[r];
+        off[r] = c0 + r < a.Cq ? a.key_offsets[(size_t)bh * a.Cq + c0 + r] : 0;
+    }
+    for (int j0 = 0; j0 < a.N; j0 += NT) {
+        const int j = j0 + tid;
+        bool sel[R], tie[R];
+        if (j < a.N) {
+            uint32_t code = __ldg(codes + j);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                uint32_t key = order_key(proxy_raw(lrt[r], code));
+                sel[r] = key > tk[r];
+                tie[r] = key == tk[r];
+            }
+        } else {
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                sel[r] = tie[r] = false;
+        }
+        uint32_t bs[R], bt[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            bs[r] = __ballot_sync(0xffffffffu, sel[r]);
+            bt[r] = __ballot_sync(0xffffffffu, tie[r]);
+            if (lane == 0) {
+                wsel[r][warp] = __popc(bs[r]);
+                wtie[r][warp] = __popc(bt[r]);
+            }
+        }
+        __syncthreads();
+        // exclusive prefix over warps: warp (2r + q) scans row r, quantity q
+        if (warp < 2 * R) {
+            int r = warp >> 1, q = warp & 1;
+            int *arr = q ? wtie[r] : wsel[r];
+            int v = lane < NWARP ? arr[lane] : 0;
+            int inc = v;
+            for (int o = 1; o < 32; o <<= 1) {
+                int u = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o)
+                    inc += u;
+            }
+            int *base = q ? &base_tie[r] : &base_sel[r];
+            int b = *base;
+            __syncwarp();
+            if (lane < NWARP)
+                arr[lane] = b + inc - v;
+            if (lane == 31)
+                *base = b + inc;
+        }
+        __syncthreads();
+        const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            if (sel[r] || tie[r]) {
+                int sb = wsel[r][warp] + __popc(bs[r] & lt);
+                int tb = wtie[r][warp] + __popc(bt[r] & lt);
+                if (sel[r] || tb < nd[r])
+                    a.key_indices[off[r] + sb + min(tb, nd[r])] = j;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+}  // namespace
+
+static size_t topp_smem(const SelectArgs &a)
+{
+    return (size_t)R * NB * (sizeof(double) + sizeof(uint32_t)) + (size_t)R * (a.Ct + a.Ch + a.Cw) * sizeof(float);
+}
+static size_t emit_smem(const SelectArgs &a)
+{
+    return (size_t)R * NB * sizeof(uint32_t) + (size_t)R * (a.Ct + a.Ch + a.Cw) * sizeof(float);
+}
+
+void launch_select(const SelectArgs &a, cudaStream_t st)
+{
+    cudaFuncSetAttribute(select_topp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topp_smem(a));
+    cudaFuncSetAttribute(select_emit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)emit_smem(a));
+    dim3 grid((a.Cq + R - 1) / R, a.BH);
+    select_topp_kernel<<<grid, NT, topp_smem(a), st>>>(a);
+    khead_kernel<<<1, 1024, 0, st>>>(a);
+    select_emit_kernel<<<grid, NT, emit_smem(a), st>>>(a);
+    count_launch(3);
+}
+
+}  // namespace scope

@@ -1,0 +1,293 @@
+"""CUDA path vs the CPU oracle, element by element, through the C ABI.
+
+Integer results (labels, codes, counts, per-head k, key sets, query grouping) must be
+bit-exact; centroids and score tables, which are fp64 accumulations rounded once on
+both sides, must be bit-identical as well; the attention output (bf16 in, fp32
+accumulate, bf16 out) must stay within max-abs 2e-2 and relative L2 1e-2 of the fp32
+oracle.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import scope_oracle as orc
+from paper_2608_12780_b200 import binding as sb
+from paper_2608_12780_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+ATTN_MAX_ABS = 2e-2
+ATTN_REL_L2 = 1e-2
+
+
+def _dev(u16):
+    return sb.bits_to_torch(u16, device="cuda")
+
+
+def _layer(cfg, seed):
+    Q, K, V = inputs.make_qkv(cfg, seed)
+    return Q, K, V, _dev(Q), _dev(K), _dev(V)
+
+
+def _oracle_plans(Q, K, cfg):
+    return orc.plan_layer(Q, K, cfg, threads=8)
+
+
+def _key_sets(plan, bh, Cq):
+    off = plan.export("KEY_OFFSETS")
+    idx = plan.export("KEY_INDICES")
+    return [idx[off[bh * Cq + c]: off[bh * Cq + c + 1]] for c in range(Cq)]
+
+
+def _compare_plan(plan, ref, cfg, what=("kmeans", "lut", "select", "group")):
+    BH, Cq = len(ref), cfg.Cq
+    if "kmeans" in what:
+        g = plan.export("Q_ASSIGN")
+        qc = plan.export("Q_CENTROIDS")
+        nc = plan.export("CLUSTER_SIZES")
+        z = [plan.export(f"K_CODES_{m}") for m in "THW"]
+        u = [plan.export(f"K_CENTROIDS_{m}") for m in "THW"]
+        for bh in range(BH):
+            assert np.array_equal(g[bh], ref[bh].g), f"query labels, head {bh}"
+            assert np.array_equal(nc[bh], ref[bh].n_c)
+            assert np.array_equal(qc[bh], ref[bh].Qbar), f"query centroids, head {bh}"
+            for m in range(3):
+                assert np.array_equal(z[m][bh], ref[bh].z[m]), f"key codes {m}, head {bh}"
+                assert np.array_equal(u[m][bh], ref[bh].U[m]), f"key centroids {m}, head {bh}"
+    if "lut" in what:
+        for m, name in enumerate("THW"):
+            P = plan.export(f"LUT_{name}")
+            for bh in range(BH):
+                assert np.array_equal(P[bh], ref[bh].P[m]), f"table {name}, head {bh}"
+    if "select" in what:
+        t, b, r, k = (plan.export(n) for n in ("TOPP_COUNT", "BASE_COUNT", "FINAL_COUNT", "K_HEAD"))
+        off = plan.export("KEY_OFFSETS")
+        idx = plan.export("KEY_INDICES")
+        for bh in range(BH):
+            assert np.array_equal(t[bh], ref[bh].t_c), f"t_c, head {bh}: {t[bh]} vs {ref[bh].t_c}"
+            assert np.array_equal(b[bh], ref[bh].b_c)
+            assert k[bh] == ref[bh].k_head
+            assert np.array_equal(r[bh], ref[bh].r_c)
+            for c in range(Cq):
+                S = idx[off[bh * Cq + c]: off[bh * Cq + c + 1]]
+                assert np.array_equal(S, ref[bh].S[c]), f"key set, head {bh} cluster {c}"
+        assert off[0] == 0 and off[-1] == sum(int(p.r_c.sum()) for p in ref)
+    if "group" in what:
+        perm, qoff = plan.export("Q_PERM"), plan.export("Q_OFFSETS")
+        for bh in range(BH):
+            assert np.array_equal(qoff[bh], np.concatenate([[0], np.cumsum(ref[bh].n_c)]))
+            assert np.array_equal(perm[bh], np.argsort(ref[bh].g, kind="stable"))
+
+
+def _attn_errors(O_gpu, ref):
+    o = O_gpu.astype(np.float64)
+    err = np.abs(o - ref).max()
+    rel = np.linalg.norm(o - ref) / np.linalg.norm(ref)
+    return err, rel
+
+
+def _to_np(t):
+    return t.detach().float().cpu().numpy()
+
+
+@pytest.mark.parametrize("name,seed", [("tiny", 0), ("tiny", 1), ("small", 0)])
+def test_plan_end_to_end_bit_exact(name, seed):
+    cfg = inputs.CONFIGS[name]
+    Q, K, V, dQ, dK, dV = _layer(cfg, seed)
+    ref = _oracle_plans(Q, K, cfg)
+    # the decisions must be well away from a coin toss for "bit-exact" to be a fair demand
+    assert min(p.kmeans_gap for p in ref) > 1e-9 and min(p.topp_margin for p in ref) > 1e-11
+    plan = sb.Plan(sb.make_params(cfg))
+    sb.scope_plan(dQ, dK, plan)
+    plan.check()
+    _compare_plan(plan, ref, cfg)
+
+
+@pytest.mark.parametrize("name,seed", [("tiny", 0), ("small", 1)])
+def test_forward_matches_oracle(name, seed):
+    cfg = inputs.CONFIGS[name]
+    Q, K, V, dQ, dK, dV = _layer(cfg, seed)
+    plan = sb.Plan(sb.make_params(cfg))
+    O = sb.scope_forward(dQ, dK, dV, plan)
+    plan.check()
+    O = _to_np(O)
+    for h in range(cfg.H):
+        Oref, _ = orc.forward_head(Q[0, h], K[0, h], V[0, h], cfg)
+        err, rel = _attn_errors(O[0, h], Oref)
+        assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (h, err, rel)
+
+
+def test_kmeans_teacher_forced_single_iterations():
+    """Each Lloyd iteration on its own, started from the oracle's centroids of the iteration before."""
+    cfg = inputs.CONFIGS["small"]
+    Q, K, V, dQ, dK, dV = _layer(cfg, 2)
+    one = cfg.replace(iters=1)
+    plan = sb.Plan(sb.make_params(one))
+    ranges = ((0, cfg.split[0], cfg.Ct), (cfg.split[0], cfg.split[1], cfg.Ch), (cfg.split[0] + cfg.split[1], cfg.split[2], cfg.Cw))
+    for it in range(3):
+        if it == 0:
+            sb.scope_plan_stages(dQ, dK, plan, sb.STAGE_KMEANS_INIT)
+        else:
+            qc = np.stack([orc.kmeans(Q[0, h], 0, cfg.d, cfg.Cq, it).U for h in range(cfg.H)])
+            plan.import_("Q_CENTROIDS", qc)
+            for (ch0, D, Cn), m in zip(ranges, "THW"):
+                plan.import_(f"K_CENTROIDS_{m}", np.stack([orc.kmeans(K[0, h], ch0, D, Cn, it).U for h in range(cfg.H)]))
+            # imported centroids need their norms: a zero-iteration pass does not exist, so
+            # the library recomputes them at the start of every stage call
+        sb.scope_plan_stages(dQ, dK, plan, sb.STAGE_KMEANS_Q | sb.STAGE_KMEANS_K)
+        g = plan.export("Q_ASSIGN")
+        qc = plan.export("Q_CENTROIDS")
+        for h in range(cfg.H):
+            r = orc.kmeans(Q[0, h], 0, cfg.d, cfg.Cq, it + 1)
+            assert np.array_equal(g[h], r.assign), (it, h)
+            assert np.array_equal(qc[h], r.U), (it, h)
+        for (ch0, D, Cn), m in zip(ranges, "THW"):
+            z = plan.export(f"K_CODES_{m}")
+            u = plan.export(f"K_CENTROIDS_{m}")
+            for h in range(cfg.H):
+                r = orc.kmeans(K[0, h], ch0, D, Cn, it + 1)
+                assert np.array_equal(z[h], r.assign), (it, m, h)
+                assert np.array_equal(u[h], r.U), (it, m, h)
+
+
+def _import_upstream(plan, ref, upto):
+    """Feed the oracle's arrays of the stages before `upto` into the plan."""
+    st = lambda f: np.stack([f(p) for p in ref])
+    plan.import_("Q_CENTROIDS", st(lambda p: p.Qbar))
+    for m, name in enumerate("THW"):
+        plan.import_(f"K_CENTROIDS_{name}", st(lambda p: p.U[m]))
+        plan.import_(f"K_CODES_{name}", st(lambda p: p.z[m]))
+    plan.import_("Q_ASSIGN", st(lambda p: p.g))
+    plan.import_("CLUSTER_SIZES", st(lambda p: p.n_c))
+    if upto in ("select", "attn"):
+        for m, name in enumerate("THW"):
+            plan.import_(f"LUT_{name}", st(lambda p: p.P[m]))
+    if upto == "attn":
+        Cq = ref[0].n_c.shape[0]
+        plan.import_("FINAL_COUNT", st(lambda p: p.r_c))
+        sizes = np.concatenate([p.r_c for p in ref]).astype(np.int64)
+        plan.import_("KEY_OFFSETS", np.concatenate([[0], np.cumsum(sizes)]))
+        plan.import_("KEY_INDICES", np.concatenate([np.concatenate(p.S) for p in ref]))
+        plan.import_("Q_PERM", st(lambda p: np.argsort(p.g, kind="stable")))
+        plan.import_("Q_OFFSETS", st(lambda p: np.concatenate([[0], np.cumsum(p.n_c)])))
+
+
+@pytest.mark.parametrize("name,seed", [("tiny", 3), ("small", 3)])
+def test_stages_teacher_forced(name, seed):
+    cfg = inputs.CONFIGS[name]
+    Q, K, V, dQ, dK, dV = _layer(cfg, seed)
+    ref = _oracle_plans(Q, K, cfg)
+    plan = sb.Plan(sb.make_params(cfg))
+    _import_upstream(plan, ref, "lut")
+    sb.scope_plan_stages(None, None, plan, sb.STAGE_LUT)
+    _compare_plan(plan, ref, cfg, what=("lut",))
+    _import_upstream(plan, ref, "select")
+    sb.scope_plan_stages(None, None, plan, sb.STAGE_SELECT | sb.STAGE_GROUP)
+    plan.check()
+    _compare_plan(plan, ref, cfg, what=("select", "group"))
+    # attention from a fully imported plan
+    plan2 = sb.Plan(sb.make_params(cfg))
+    _import_upstream(plan2, ref, "attn")
+    O = _to_np(sb.scope_sparse_attn(dQ, dK, dV, plan2))
+    for h in range(cfg.H):
+        rows = np.arange(cfg.N)
+        Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], ref[h].g, ref[h].S, cfg.scale, rows)
+        err, rel = _attn_errors(O[0, h], Oref)
+        assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (h, err, rel)
+
+
+def test_rho_one_and_dense_mode_equal_dense_attention():
+    cfg = inputs.CONFIGS["tiny"].replace(top_p=1.0)
+    Q, K, V, dQ, dK, dV = _layer(cfg, 4)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.H * cfg.Cq * cfg.N))
+    O = _to_np(sb.scope_forward(dQ, dK, dV, plan))
+    plan.check()
+    assert np.all(plan.export("FINAL_COUNT") == cfg.N)
+    Od = _to_np(sb.scope_dense_attn(dQ, dK, dV, plan))
+    for h in range(cfg.H):
+        ref = orc.dense_rows(Q[0, h], K[0, h], V[0, h], cfg.scale, np.arange(cfg.N))
+        for o in (O[0, h], Od[0, h]):
+            err, rel = _attn_errors(o, ref)
+            assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2
+
+
+def test_ragged_shapes_and_strides():
+    """N not a multiple of any tile, odd cluster counts, a 44/42/42 split and padded strides."""
+    cfg = inputs.ScopeConfig("ragged", 1, 3, (3, 7, 11), (44, 42, 42), 13, 5, 9, 7, 4, 0.85, 17)
+    Q, K, V = inputs.make_qkv(cfg, 7)
+    N, d, H = cfg.N, cfg.d, cfg.H
+    sn, sh = d + 64, (N + 3) * (d + 64)
+    def padded(u16):
+        buf = torch.zeros(1, H, N + 3, d + 64, dtype=torch.bfloat16, device="cuda")
+        buf[:, :, :N, :d] = _dev(u16)
+        return buf
+    bQ, bK, bV = padded(Q), padded(K), padded(V)
+    bO = torch.zeros_like(bQ)
+    params = sb.make_params(cfg, strides=(H * sh, sh, sn))
+    plan = sb.Plan(params)
+    sb.scope_forward(bQ, bK, bV, plan, bO)
+    plan.check()
+    ref = _oracle_plans(Q, K, cfg)
+    _compare_plan(plan, ref, cfg)
+    O = _to_np(bO)[0, :, :N, :d]
+    assert np.all(_to_np(bO)[0, :, N:, :] == 0) and np.all(_to_np(bO)[0, :, :, d:] == 0)
+    for h in range(H):
+        Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], ref[h].g, ref[h].S, cfg.scale, np.arange(N))
+        err, rel = _attn_errors(O[h], Oref)
+        assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2
+
+
+def test_degenerate_cluster_counts():
+    """One cluster everywhere; and one cluster per token."""
+    base = inputs.CONFIGS["tiny"].replace(H=1, grid=(2, 4, 5))
+    for cfg in (base.replace(Cq=1, Ct=1, Ch=1, Cw=1, k_fix=3), base.replace(Cq=40, Ct=40, Ch=40, Cw=40, k_fix=40, iters=2)):
+        Q, K, V, dQ, dK, dV = _layer(cfg, 9)
+        plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.Cq * cfg.N))
+        O = _to_np(sb.scope_forward(dQ, dK, dV, plan))
+        plan.check()
+        ref = _oracle_plans(Q, K, cfg)
+        _compare_plan(plan, ref, cfg)
+        Oref = orc.attention_rows(Q[0, 0], K[0, 0], V[0, 0], ref[0].g, ref[0].S, cfg.scale, np.arange(cfg.N))
+        err, rel = _attn_errors(O[0, 0], Oref)
+        assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2
+
+
+def test_capacity_overflow_is_reported_not_written():
+    cfg = inputs.CONFIGS["tiny"]
+    Q, K, V, dQ, dK, dV = _layer(cfg, 0)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=64))
+    O = torch.full_like(dQ, 7.0)
+    sb.scope_forward(dQ, dK, dV, plan, O)
+    status, need = plan.status()
+    assert status == sb.SCOPE_ERR_CAPACITY and need > 64
+    assert torch.all(O == 7.0)  # attention refuses to run on a truncated plan
+    big = sb.Plan(sb.make_params(cfg, index_capacity=need))
+    sb.scope_forward(dQ, dK, dV, big, O)
+    assert big.status() == (sb.SCOPE_OK, need)
+
+
+def test_bad_imported_plan_is_rejected():
+    cfg = inputs.CONFIGS["tiny"]
+    plan = sb.Plan(sb.make_params(cfg))
+    g = np.zeros((cfg.H, cfg.N), np.int32)
+    g[1, 5] = cfg.Cq  # out of range
+    with pytest.raises(sb.ScopeError) as e:
+        plan.import_("Q_ASSIGN", g)
+    assert e.value.status == sb.SCOPE_ERR_BAD_PLAN
+    plan.reset_status()
+    off = np.arange(cfg.H * cfg.Cq + 1, dtype=np.int64)[::-1].copy()  # decreasing
+    with pytest.raises(sb.ScopeError):
+        plan.import_("KEY_OFFSETS", off)
+    plan.reset_status()
+    plan.import_("Q_ASSIGN", np.zeros((cfg.H, cfg.N), np.int32))
+    assert plan.status()[0] == sb.SCOPE_OK
+
+
+def test_repeatable_and_plan_reuse():
+    cfg = inputs.CONFIGS["small"]
+    Q, K, V, dQ, dK, dV = _layer(cfg, 5)
+    plan = sb.Plan(sb.make_params(cfg))
+    O1 = sb.scope_forward(dQ, dK, dV, plan).clone()
+    idx1 = plan.export("KEY_INDICES")
+    O2 = sb.scope_forward(dQ, dK, dV, plan)
+    assert torch.equal(O1, O2) and np.array_equal(idx1, plan.export("KEY_INDICES"))
