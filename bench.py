@@ -1,0 +1,362 @@
+"""Benchmark of the SCOPE attention layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload HY720] [--impl scope|reference]
+
+A step is one pass of the whole layer (k-means of Q and K, score tables, selection,
+query grouping, sparse attention) over one synthetic layer input per GPU.  With N > 1
+(launched by torchrun, one process per GPU) every rank runs its own layer of a batch of
+N: the path has no exchange step, so scaling is weak and there is no collective in the
+timed region besides the bracketing barrier.  Rank 0 prints one JSON line.
+
+--impl reference times the CPU oracle (the plain restatement of the paper used by the
+tests) on the host cores, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_12780_b200 import inputs  # noqa: E402
+
+METRIC = "SCOPE attn-layer ms at 118.8K tokens; sparse-attn TFLOP/s; select GB/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------------------- CPU oracle arm
+
+
+def oracle_sample(cfg, seed=0):
+    """Time the oracle, as it stands, single-threaded, on a bounded sample of one layer and
+    extrapolate to ms per layer: one Lloyd iteration of one head (queries and the three key
+    ranges), the tables, the selection of 8 query clusters and the attention of 128 query rows."""
+    from oracle import scope_oracle as orc
+
+    Q, K, V = inputs.make_head(cfg, seed, 0, 0)
+    N, d = cfg.N, cfg.d
+    it_s = min(2, cfg.iters)
+    t0 = time.perf_counter()
+    kq = orc.kmeans(Q, 0, d, cfg.Cq, it_s)
+    ranges = ((0, cfg.split[0], cfg.Ct), (cfg.split[0], cfg.split[1], cfg.Ch), (cfg.split[0] + cfg.split[1], cfg.split[2], cfg.Cw))
+    ks = [orc.kmeans(K, ch0, D, Cn, it_s) for ch0, D, Cn in ranges]
+    t_iter = (time.perf_counter() - t0) / it_s
+    t0 = time.perf_counter()
+    P = tuple(orc.lut(kq.U, ch0, km.U)[0] for (ch0, _, _), km in zip(ranges, ks))
+    t_lut = time.perf_counter() - t0
+    z = tuple(km.assign for km in ks)
+    rows_sel = min(16, cfg.Cq)
+    t0 = time.perf_counter()
+    orders, b = [], []
+    for c in range(rows_sel):
+        raw = orc.scores_row(P[0][c], P[1][c], P[2][c], *z)
+        o, tc, _ = orc.topp_row(raw, cfg.scale, cfg.top_p)
+        orders.append(o)
+        b.append(max(tc, cfg.k_fix))
+    # per-head k from the sampled clusters (Eq. 9 with their sizes), then Eq. 10
+    n_s = kq.counts[:rows_sel].astype(np.int64)
+    k_est = int(-(-int((n_s * np.array(b)).sum()) // max(1, int(n_s.sum()))))
+    r = [min(N, max(bc, k_est)) for bc in b]
+    S = [orc.key_set(orders[c], r[c]) for c in range(rows_sel)]
+    t_sel = time.perf_counter() - t0
+    rows_att = min(128, N)
+    g = (np.arange(N) % rows_sel).astype(np.int32)
+    t0 = time.perf_counter()
+    orc.attention_rows(Q, K, V, g, S, cfg.scale, np.arange(rows_att))
+    t_att = time.perf_counter() - t0
+    per_head = cfg.iters * t_iter + t_lut + t_sel * cfg.Cq / rows_sel + t_att * N / rows_att
+    ms_layer = 1e3 * per_head * cfg.H
+    sample = (f"1 of {cfg.H} heads: {it_s} of {cfg.iters} Lloyd iterations (Q and 3 key ranges), tables, selection of "
+              f"{rows_sel}/{cfg.Cq} query clusters, attention of {rows_att}/{N} rows over their key sets "
+              f"(mean {int(np.mean(r))} keys); scaled to one layer; measured "
+              f"{t_iter * it_s + t_lut + t_sel + t_att:.1f} s")
+    return ms_layer, sample
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for _ in range(args.warmup):
+        pass  # the oracle has no warm-up state worth paying for
+    sample = ""
+    for _ in range(max(1, args.steps)):
+        ms, sample = oracle_sample(cfg)
+        vals.append(ms)
+    ms = float(np.median(vals))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": ms, "unit": "ms/layer", "n_gpus": args.gpus,
+        "steps": max(1, args.steps), "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "tokens": cfg.N, "heads": cfg.H},
+        "cpu_baseline": {"value": ms, "unit": "ms/layer", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": ms, "unit": "ms/layer", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------- clocks
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                       "-lms", "50", "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.f:
+            tok = [t.strip() for t in line.split(",")]
+            if len(tok) < 7:
+                continue
+            try:
+                sm.append(float(tok[0]))
+                mx.append(float(tok[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, tok[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# --------------------------------------------------------------------------------------- CUDA arm
+
+
+def run_scope(args, cfg):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_12780_b200 import binding as sb
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    sb.lib()  # fail loudly before any work if the library is missing
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # one layer per rank: batch element `rank` of a batch of `world`
+    nbytes = cfg.H * cfg.N * cfg.d * 2
+    host = [torch.empty((1, cfg.H, cfg.N, cfg.d), dtype=torch.bfloat16).pin_memory() for _ in range(4)]
+    views = tuple(h.view(torch.int16).numpy().view(np.uint16) for h in host[:3])
+    inputs.make_qkv(cfg, seed=args.seed, threads=args.gen_threads, batch_offset=rank, out=views)
+    dQ, dK, dV = (h.to(dev, non_blocking=True) for h in host[:3])
+    dO = torch.empty_like(dQ)
+    plan = sb.Plan(sb.make_params(cfg), device=dev)
+    torch.cuda.synchronize()
+
+    stream = torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def step(e_mid=None):
+        sb.scope_plan(dQ, dK, plan)
+        if e_mid is not None:
+            e_mid[0].record(stream)
+        sb.scope_sparse_attn(dQ, dK, dV, plan, dO)
+        if e_mid is not None:
+            e_mid[1].record(stream)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    need = plan.check("warm-up")
+
+    # ---- timed region: K steps, device-resident inputs (3 x %d MB per layer: larger than L2)
+    mids = [(ev(), ev()) for _ in range(args.steps)]
+    e0, e1 = ev(), ev()
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = sb.scope_kernel_launches()
+    barrier()
+    e0.record(stream)
+    for k in range(args.steps):
+        step(mids[k])
+    e1.record(stream)
+    barrier()
+    launches = sb.scope_kernel_launches() - launches0
+    clocks = sampler.stop() if sampler else None
+    plan.check("timed region")
+    ms_total = e0.elapsed_time(e1)
+    attn_ms = float(np.mean([m[0].elapsed_time(m[1]) for m in mids]))
+    t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+
+    # ---- plan statistics (selected pairs = the attention kernel's algorithmic work)
+    n_c = plan.export("CLUSTER_SIZES").astype(np.int64)
+    r_c = plan.export("FINAL_COUNT").astype(np.int64)
+    t_c = plan.export("TOPP_COUNT").astype(np.int64)
+    b_c = plan.export("BASE_COUNT").astype(np.int64)
+    k_head = plan.export("K_HEAD")
+    pairs = int((n_c * r_c).sum())
+    attn_flop = 4.0 * cfg.d * pairs
+    density = pairs / (cfg.H * cfg.N * cfg.N)
+
+    # ---- per-stage times (outside the timed region)
+    def time_stage(fn, reps=3):
+        ts = []
+        for _ in range(reps):
+            a, b = ev(), ev()
+            torch.cuda.synchronize()
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return float(np.median(ts))
+
+    stage_ms = {
+        "kmeans_q": time_stage(lambda: sb.scope_plan_stages(dQ, dK, plan, sb.STAGE_KMEANS_INIT | sb.STAGE_KMEANS_Q)),
+        "kmeans_k": time_stage(lambda: sb.scope_plan_stages(dQ, dK, plan, sb.STAGE_KMEANS_INIT | sb.STAGE_KMEANS_K)),
+    }
+    sb.scope_plan_stages(dQ, dK, plan, sb.STAGE_KMEANS_INIT | sb.STAGE_KMEANS_Q | sb.STAGE_KMEANS_K)
+    stage_ms["lut"] = time_stage(lambda: sb.scope_plan_stages(None, None, plan, sb.STAGE_LUT))
+    stage_ms["select"] = time_stage(lambda: sb.scope_plan_stages(None, None, plan, sb.STAGE_SELECT))
+    stage_ms["group"] = time_stage(lambda: sb.scope_plan_stages(None, None, plan, sb.STAGE_GROUP))
+    stage_ms["sparse_attn"] = time_stage(lambda: sb.scope_sparse_attn(dQ, dK, dV, plan, dO))
+
+    # ---- dense comparator: Eq. 1 through the same kernel on a few heads, scaled to the layer
+    dense_ms = None
+    if args.dense_heads > 0 and rank == 0:
+        hh = min(args.dense_heads, cfg.H)
+        sub = sb.make_params(cfg, H=hh, strides=(cfg.H * cfg.N * cfg.d, cfg.N * cfg.d, cfg.d), index_capacity=1)
+        dplan = sb.Plan(sub, device=dev)
+        sb.scope_dense_attn(dQ, dK, dV, dplan, dO)
+        dense_ms = time_stage(lambda: sb.scope_dense_attn(dQ, dK, dV, dplan, dO), reps=2) * cfg.H / hh
+        del dplan
+
+    # ---- end to end through the host entry point: pinned host tensors in, pinned host tensor out
+    e2e = None
+    if args.e2e_steps > 0:
+        staging = torch.empty(4 * nbytes + 512, dtype=torch.uint8, device=dev)
+        sb.scope_forward_host(host[0], host[1], host[2], plan, host[3], staging)
+        barrier()
+        a, b = ev(), ev()
+        a.record(stream)
+        for _ in range(args.e2e_steps):
+            sb.scope_forward_host(host[0], host[1], host[2], plan, host[3], staging)
+        b.record(stream)
+        barrier()
+        te = torch.tensor([a.elapsed_time(b)], device=dev, dtype=torch.float64)
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e2e = {"value": float(te.item()) / args.e2e_steps / world, "unit": "ms/layer",
+               "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes, "steps": args.e2e_steps}
+        del staging
+
+    if rank == 0:
+        peaks = measured_peaks()
+        achieved = attn_flop / (attn_ms * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"]
+        sel_bytes = cfg.H * cfg.N * 4 + int(r_c.sum()) * 4  # codes in, index lists out (algorithmic)
+        line = {
+            "metric": METRIC, "value": ms_step / world, "unit": "ms/layer", "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "tokens": cfg.N, "heads": cfg.H, "head_dim": cfg.d, "split": list(cfg.split),
+                       "Cq": cfg.Cq, "C_thw": [cfg.Ct, cfg.Ch, cfg.Cw], "kmeans_iters": cfg.iters, "top_p": cfg.top_p,
+                       "k_fix": cfg.k_fix, "layers_per_gpu": 1, "parallelism": f"batch-sharded x{world}, no collective",
+                       "l2": "inputs larger than L2 (Q, K, V %d MB each)" % (nbytes >> 20)},
+            "roofline": {"bound": "tensor", "kernel": "sparse_attn_kernel", "achieved": achieved, "peak": peak,
+                         "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                         "peak_source": f"bf16_tflops_sustained of {peaks['source']}",
+                         "flop_per_launch": attn_flop, "ms_per_launch": attn_ms},
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "stage_ms": stage_ms,
+            "sparse_attn_tflops": achieved,
+            "select_gbs": sel_bytes / (stage_ms["select"] * 1e-3) / 1e9,
+            "kmeans_gbs": cfg.iters * 2 * nbytes / ((stage_ms["kmeans_q"] + stage_ms["kmeans_k"]) * 1e-3) / 1e9,
+            "dense_attn_ms_same_kernel": dense_ms,
+            "plan_stats": {"density": density, "selected_pairs": pairs, "index_entries": int(need),
+                           "k_head_min_med_max": [int(k_head.min()), int(np.median(k_head)), int(k_head.max())],
+                           "t_c_min_med_max": [int(t_c.min()), int(np.median(t_c)), int(t_c.max())],
+                           "r_c_min_med_max": [int(r_c.min()), int(np.median(r_c)), int(r_c.max())],
+                           "clusters_extended_frac": float((b_c < r_c).mean()),
+                           "floor_binding_frac": float((t_c < b_c).mean())},
+        }
+        if args.cpu_baseline:
+            ms_cpu, sample = oracle_sample(cfg, args.seed)
+            line["cpu_baseline"] = {"value": ms_cpu, "unit": "ms/layer", "cores": 1, "kind": "oracle", "sample": sample}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="scope", choices=["scope", "reference"])
+    ap.add_argument("--workload", default="HY720", choices=sorted(inputs.CONFIGS))
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--gen-threads", type=int, default=min(16, os.cpu_count() or 1))
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--dense-heads", type=int, default=1)
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--heads", type=int, default=0, help="profiling only: run a subset of the workload's heads")
+    args = ap.parse_args()
+    cfg = inputs.CONFIGS[args.workload]
+    if args.heads > 0:
+        cfg = cfg.replace(H=args.heads, name=f"{cfg.name}[{args.heads} heads]")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != max(1, args.gpus) and world > 1:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_scope(args, cfg)
+
+
+if __name__ == "__main__":
+    main()
