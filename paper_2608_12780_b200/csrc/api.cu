@@ -29,6 +29,7 @@ struct scope_plan_s {
     int32_t *q_perm, *q_offsets;
     // scratch
     float *q_unorm, *k_unorm[3], *q_u2max, *k_u2max[3];
+    bf16 *q_split, *k_split[3];
     double *q_sums, *k_sums[3];
     int32_t *q_counts, *k_counts[3];
     RowState *rows;
@@ -107,12 +108,14 @@ void carve(scope_plan_t *pl, unsigned char *base, size_t *total)
     pl->q_u2max = cv.take<float>(BH);
     pl->q_sums = cv.take<double>(BH * Cq * p.d);
     pl->q_counts = cv.take<int32_t>(BH * Cq);
+    pl->q_split = cv.take<bf16>(BH * 3 * ((Cq + 15) & ~(size_t)15) * p.d);
     for (int m = 0; m < 3; ++m) {
         pl->k_cent[m] = cv.take<float>(BH * C[m] * D[m]);
         pl->k_unorm[m] = cv.take<float>(BH * C[m]);
         pl->k_u2max[m] = cv.take<float>(BH);
         pl->k_sums[m] = cv.take<double>(BH * C[m] * D[m]);
         pl->k_counts[m] = cv.take<int32_t>(BH * C[m]);
+        pl->k_split[m] = cv.take<bf16>(BH * 3 * ((C[m] + 15) & ~(size_t)15) * p.d);
         pl->lut[m] = cv.take<float>(BH * Cq * C[m]);
     }
     pl->q_assign = cv.take<int32_t>(BH * N);
@@ -153,7 +156,8 @@ KmArgs q_args(const scope_plan_t *pl, const void *Q)
     a.sb = p.stride_b; a.sh = p.stride_h; a.sn = p.stride_n;
     a.B = p.B; a.H = p.H; a.N = p.N;
     a.nspaces = 1;
-    a.sp[0] = KmSpace{0, p.d, p.Cq, pl->q_cent, pl->q_unorm, pl->q_u2max, pl->q_sums, pl->q_counts, pl->n_c};
+    a.sp[0] = KmSpace{0, p.d, p.Cq, pl->q_cent, pl->q_unorm, pl->q_u2max, pl->q_sums, pl->q_counts, pl->n_c,
+                      pl->q_split, (p.Cq + 15) & ~15};
     a.assign = pl->q_assign;
     a.codes = nullptr;
     return a;
@@ -170,7 +174,7 @@ KmArgs k_args(const scope_plan_t *pl, const void *K)
     const int ch0[3] = {0, p.d_t, p.d_t + p.d_h}, D[3] = {p.d_t, p.d_h, p.d_w}, C[3] = {p.Ct, p.Ch, p.Cw};
     for (int m = 0; m < 3; ++m)
         a.sp[m] = KmSpace{ch0[m], D[m], C[m], pl->k_cent[m], pl->k_unorm[m], pl->k_u2max[m], pl->k_sums[m],
-                          pl->k_counts[m], nullptr};
+                          pl->k_counts[m], nullptr, pl->k_split[m], (C[m] + 15) & ~15};
     a.assign = nullptr;
     a.codes = pl->k_codes;
     return a;
@@ -333,14 +337,14 @@ scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, u
         if (!(stages & SCOPE_STAGE_KMEANS_INIT))
             launch_kmeans_norms(a, st);  // centroids may have been imported
         for (int it = 0; it < p.kmeans_iters; ++it)
-            launch_kmeans_iteration(a, st);
+            launch_kmeans_iteration(a, pl->status, st);
     }
     if (stages & SCOPE_STAGE_KMEANS_K) {
         KmArgs a = k_args(pl, K);
         if (!(stages & SCOPE_STAGE_KMEANS_INIT))
             launch_kmeans_norms(a, st);
         for (int it = 0; it < p.kmeans_iters; ++it)
-            launch_kmeans_iteration(a, st);
+            launch_kmeans_iteration(a, pl->status, st);
     }
     if (stages & SCOPE_STAGE_LUT) {
         KmArgs a = k_args(pl, K);

@@ -10,6 +10,8 @@
 // plain sum of squared differences in fp64, channel by channel, lowest index winning a
 // tie.  Member sums are accumulated in fp64 (sums of bf16 values are exact there, so their
 // order does not matter) and rounded once to fp32 after the division.
+#include <cstdlib>
+
 #include "scope_internal.cuh"
 
 namespace scope {
@@ -311,6 +313,21 @@ __global__ void __launch_bounds__(256) kmeans_finalize_kernel(KmArgs a, int mode
         sums[e] = 0.0;
     }
     __syncthreads();
+    if (sp.split) {
+        // u = hi + mid + lo in bf16 (exact to 24 bits), laid out over absolute channels
+        bf16 *split = sp.split + (size_t)bh * 3 * sp.cpad * kHeadDim;
+        for (int e = threadIdx.x; e < sp.cpad * kHeadDim; e += blockDim.x) {
+            int r = e / kHeadDim, ch = e % kHeadDim;
+            float u = (r < sp.C && ch >= sp.ch0 && ch < sp.ch0 + sp.D) ? cent[(size_t)r * sp.D + (ch - sp.ch0)] : 0.f;
+            bf16 hi = __float2bfloat16_rn(u);
+            float r1 = u - __bfloat162float(hi);
+            bf16 mid = __float2bfloat16_rn(r1);
+            bf16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+            split[e] = hi;
+            split[(size_t)sp.cpad * kHeadDim + e] = mid;
+            split[(size_t)2 * sp.cpad * kHeadDim + e] = lo;
+        }
+    }
     float mx = 0.f;
     for (int r = threadIdx.x; r < sp.C; r += blockDim.x) {
         float n2 = 0.f;
@@ -349,13 +366,19 @@ void launch_kmeans_norms(const KmArgs &a, cudaStream_t st)
     count_launch();
 }
 
-void launch_kmeans_iteration(const KmArgs &a, cudaStream_t st)
+void launch_kmeans_iteration(const KmArgs &a, int32_t *status, cudaStream_t st)
 {
-    dim3 grid((a.N + TM - 1) / TM, a.B * a.H);
-    kmeans_assign_kernel<<<grid, NT, 0, st>>>(a);
+    const char *force = getenv("SCOPE_KMEANS_SIMT");  // testing aid: run the general kernel
+    if (kmeans_tc_supported(a, nullptr) && !(force && force[0] == '1')) {
+        launch_kmeans_assign_tc(a, status, st);
+    } else {
+        dim3 grid((a.N + TM - 1) / TM, a.B * a.H);
+        kmeans_assign_kernel<<<grid, NT, 0, st>>>(a);
+        count_launch();
+    }
     dim3 fgrid(a.B * a.H, a.nspaces);
     kmeans_finalize_kernel<<<fgrid, 256, 0, st>>>(a, 0);
-    count_launch(2);
+    count_launch();
 }
 
 }  // namespace scope

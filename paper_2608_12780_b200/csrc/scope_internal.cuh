@@ -28,6 +28,9 @@ struct KmSpace {
     double *sums;     // [BH, C, D]  member sums of the running iteration
     int32_t *counts;  // [BH, C]
     int32_t *sizes;   // [BH, C] or null: copy of the member counts of the last assignment
+    bf16 *split;      // [BH, 3, cpad, 128] centroids as three bf16 terms over absolute channels (zero outside
+                      // the range and past C), or null
+    int cpad;         // C rounded up to a multiple of 16
 };
 
 struct KmArgs {
@@ -90,7 +93,9 @@ struct AttnArgs {
 // launchers (each enqueues on `st` and bumps the launch counter)
 void launch_kmeans_init(const KmArgs &a, cudaStream_t st);
 void launch_kmeans_norms(const KmArgs &a, cudaStream_t st);
-void launch_kmeans_iteration(const KmArgs &a, cudaStream_t st);
+void launch_kmeans_iteration(const KmArgs &a, int32_t *status, cudaStream_t st);
+bool kmeans_tc_supported(const KmArgs &a, size_t *smem_bytes);
+void launch_kmeans_assign_tc(const KmArgs &a, int32_t *status, cudaStream_t st);
 void launch_lut(int BH, int Cq, int d, const float *qcent, const KmSpace *ksp /*3*/, float *const *lut,
                 cudaStream_t st);
 void launch_select(const SelectArgs &a, cudaStream_t st);

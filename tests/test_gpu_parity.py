@@ -291,3 +291,33 @@ def test_repeatable_and_plan_reuse():
     idx1 = plan.export("KEY_INDICES")
     O2 = sb.scope_forward(dQ, dK, dV, plan)
     assert torch.equal(O1, O2) and np.array_equal(idx1, plan.export("KEY_INDICES"))
+
+
+def test_kmeans_general_kernel_path(monkeypatch):
+    """The plain fp32 assignment kernel (used when a codebook does not fit the tensor-core kernel's
+    shared memory) must reach the same labels and centroids."""
+    monkeypatch.setenv("SCOPE_KMEANS_SIMT", "1")
+    cfg = inputs.CONFIGS["small"]
+    Q, K, V, dQ, dK, dV = _layer(cfg, 6)
+    ref = _oracle_plans(Q, K, cfg)
+    plan = sb.Plan(sb.make_params(cfg))
+    before = sb.scope_kernel_launches()
+    sb.scope_plan(dQ, dK, plan)
+    plan.check()
+    _compare_plan(plan, ref, cfg)
+    monkeypatch.delenv("SCOPE_KMEANS_SIMT")
+    plan2 = sb.Plan(sb.make_params(cfg))
+    sb.scope_plan(dQ, dK, plan2)
+    plan2.check()
+    _compare_plan(plan2, ref, cfg)
+
+
+def test_large_codebooks_use_general_kernel():
+    """More centroids than the tensor-core kernel holds (C > 256): still exact."""
+    cfg = inputs.ScopeConfig("bigC", 1, 1, (6, 10, 10), (16, 56, 56), 300, 8, 272, 16, 2, 0.9, 32)
+    Q, K, V, dQ, dK, dV = _layer(cfg, 8)
+    ref = _oracle_plans(Q, K, cfg)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.Cq * cfg.N))
+    sb.scope_plan(dQ, dK, plan)
+    plan.check()
+    _compare_plan(plan, ref, cfg)
