@@ -1,90 +1,95 @@
 // Sparse attention of Eq. 11 (Algorithm 1 lines 10-12): every query of cluster c attends to the
-// original keys/values listed in S_c.  Flash-style: one block owns a tile of 64 queries of one
-// cluster (gathered through the query permutation), streams the cluster's key list in tiles of
-// 64 gathered K and V rows (cp.async, double buffered, XOR-swizzled shared memory), keeps the
-// running row maximum / row sum in registers and never materialises the logits.  bf16 operands,
-// fp32 accumulation on the tensor cores, bf16 output.  With `dense` set the key list is 0..N-1
-// and the grouping is the identity, which is Eq. 1.
+// original keys/values listed in S_c.  With `dense` set the key list is 0..N-1 and the grouping is
+// the identity, which is Eq. 1.
+//
+// Flash-style, warp-specialised, on the tcgen05 tensor cores.  One block owns a tile of 128
+// queries of one cluster (gathered through the query permutation) and streams the cluster's key
+// list in tiles of 128 gathered K and V rows:
+//   * 4 producer warps gather K/V rows with 16-byte cp.async into 128-byte-swizzled shared
+//     memory, two tiles in flight;
+//   * 1 MMA warp (one thread) issues S = Q K^T (accumulator in tensor memory, double buffered)
+//     and O += P V (accumulator in tensor memory);
+//   * 4 softmax warps, one thread per query row (= TMEM lane): read S, keep the running row
+//     maximum and row sum in registers, rescale O in tensor memory when the maximum grows, write
+//     P (bf16) as the A operand of the second MMA.
+// Roles synchronise through mbarriers only; every wait is bounded and a time-out ends the block
+// with an error status instead of hanging.
 #include "scope_internal.cuh"
+#include "sm100.cuh"
 
 namespace scope {
 
+using namespace sm100;
+
 namespace {
 
-constexpr int BM = kAttnTileRows;  // query rows per block
-constexpr int BN = 64;             // keys per tile
-constexpr int NT = 128;            // 4 warps x 16 query rows
-constexpr int ROW_BYTES = kHeadDim * 2;
-constexpr int TILE_BYTES = BN * ROW_BYTES;  // 16 KB
+constexpr int BM = kAttnTileRows;  // 128 query rows per block = MMA M
+constexpr int BN = 128;            // keys per tile
+constexpr int HALF = BM * 128;     // bytes of one 64-column half of a 128-row swizzled tile
+constexpr int TILE = 2 * HALF;     // 32 KB: a [128][128] bf16 tile
+constexpr int STAGES = 2;
+constexpr int PRODUCER_THREADS = 128, SOFTMAX_THREADS = 128;
+constexpr int NT = PRODUCER_THREADS + 32 + SOFTMAX_THREADS;  // 288
+constexpr int SMEM_BYTES = 1024 + TILE /*Q*/ + STAGES * 2 * TILE /*K,V*/ + TILE /*P*/;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O = 256;
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p)
+struct Barriers {
+    uint64_t q_full;
+    uint64_t kv_full[STAGES];
+    uint64_t kv_empty[STAGES];
+    uint64_t s_full[2];
+    uint64_t s_empty[2];
+    uint64_t p_full;
+    uint64_t pv_done;
+};
+
+// bounded wait that also gives up when another role has already failed
+__device__ __forceinline__ bool wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
-    return (uint32_t)__cvta_generic_to_shared(p);
+    for (uint32_t i = 0; i < 4000000u; ++i) {
+        if (mbar_try_wait(bar, parity))
+            return true;
+        if (i > 32) {
+            __nanosleep(40);
+            if ((i & 255u) == 0 && *abort_flag)
+                return false;
+        }
+    }
+    *abort_flag = 1;
+    return false;
 }
-// byte offset of 16-byte chunk `chunk` of row `row` inside a swizzled [rows][128] bf16 tile
-__device__ __forceinline__ uint32_t swz(int row, int chunk)
-{
-    return (uint32_t)(row * ROW_BYTES + ((chunk ^ (row & 7)) << 4));
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src));
-}
-__device__ __forceinline__ void cp_async_commit()
-{
-    asm volatile("cp.async.commit_group;\n" ::);
-}
-template <int N>
-__device__ __forceinline__ void cp_async_wait()
-{
-    asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
-}
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
-{
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
-{
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
-__global__ void __launch_bounds__(NT) sparse_attn_kernel(AttnArgs a)
+__global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t *status_out)
 {
-    extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char *sQ = smem;                       // [BM][128] bf16, later the output tile
-    unsigned char *sK = smem + BM * ROW_BYTES;      // 2 stages
-    unsigned char *sV = sK + 2 * TILE_BYTES;        // 2 stages
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    unsigned char *sQ = smem;
+    unsigned char *sKV = sQ + TILE;                 // stage s: K at sKV + s*2*TILE, V right after
+    unsigned char *sP = sKV + STAGES * 2 * TILE;
+    __shared__ Barriers bars;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
 
     if (!a.dense && a.status[ST_CODE] != 0)
         return;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.y;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = bh / a.H, h = bh % a.H;
     const int64_t base = (int64_t)b * a.sb + (int64_t)h * a.sh;
     const bf16 *Qh = a.Q + base, *Kh = a.K + base, *Vh = a.V + base;
     bf16 *Oh = a.O + base;
 
-    // which cluster / which rows
-    int nrows, nkeys;
+    // which cluster / which rows (block-uniform)
+    int nrows, nkeys, row0 = 0;
     const int32_t *rowlist = nullptr;  // tokens of this tile (null: identity)
     const int32_t *keylist = nullptr;  // key indices (null: identity)
-    int row0 = 0;
     if (a.dense) {
         row0 = blockIdx.x * BM;
         if (row0 >= a.N)
@@ -115,199 +120,267 @@ __global__ void __launch_bounds__(NT) sparse_attn_kernel(AttnArgs a)
     }
     const int ntiles = (nkeys + BN - 1) / BN;
 
-    // copy roles: 16 threads per row, 8 rows per pass
-    const int crow = tid >> 4, cchunk = tid & 15;
+    if (tid == 0) {
+        s_abort = 0;
+        mbar_init(&bars.q_full, PRODUCER_THREADS);
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&bars.kv_full[s], PRODUCER_THREADS);
+            mbar_init(&bars.kv_empty[s], 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars.s_full[s], 1);
+            mbar_init(&bars.s_empty[s], SOFTMAX_THREADS);
+        }
+        mbar_init(&bars.p_full, SOFTMAX_THREADS);
+        mbar_init(&bars.pv_done, 1);
+        mbar_fence_init();
+    }
+    if (warp == 4) {
+        tmem_alloc(&s_tmem_base, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem_base;
+    volatile int *abort_flag = &s_abort;
 
-    // Q tile
-    {
-#pragma unroll
+    if (warp < 4) {
+        // ===================== producers: Q once, then K/V tiles =====================
+        const int crow = tid >> 4, cchunk = tid & 15;  // 8 rows per pass, 16 chunks per row
+        const uint32_t chunk_off = (cchunk >> 3) * HALF;
         for (int i = 0; i < BM / 8; ++i) {
             int r = crow + 8 * i;
-            int rr = min(r, nrows - 1);
-            int tok = rowlist ? rowlist[rr] : row0 + rr;
-            cp_async16(smem_u32(sQ) + swz(r, cchunk), Qh + (int64_t)tok * a.sn + cchunk * 8);
+            bool ok = r < nrows;
+            int tok = ok ? (rowlist ? rowlist[r] : row0 + r) : 0;
+            cp_async16_zfill(smem_u32(sQ) + chunk_off + sw128(r, cchunk & 7), Qh + (int64_t)tok * a.sn + cchunk * 8, ok ? 16 : 0);
         }
-    }
-    int kidx[BN / 8];
-    auto load_idx = [&](int t) {
+        cp_async_commit();
+        int kidx[BN / 8];
+        auto load_idx = [&](int t) {
 #pragma unroll
-        for (int i = 0; i < BN / 8; ++i) {
-            int j = min(t * BN + crow + 8 * i, nkeys - 1);
-            kidx[i] = keylist ? __ldg(keylist + j) : j;
-        }
-    };
-    auto issue_tile = [&](int stage) {
-        const uint32_t dk = smem_u32(sK) + stage * TILE_BYTES, dv = smem_u32(sV) + stage * TILE_BYTES;
+            for (int i = 0; i < BN / 8; ++i) {
+                int j = min(t * BN + crow + 8 * i, nkeys - 1);  // past the end: repeat the last key, masked later
+                kidx[i] = keylist ? __ldg(keylist + j) : j;
+            }
+        };
+        auto issue_tile = [&](int stage) {
+            const uint32_t dk = smem_u32(sKV) + stage * 2 * TILE + chunk_off, dv = dk + TILE;
 #pragma unroll
-        for (int i = 0; i < BN / 8; ++i) {
-            int r = crow + 8 * i;
-            const int64_t o = (int64_t)kidx[i] * a.sn + cchunk * 8;
-            cp_async16(dk + swz(r, cchunk), Kh + o);
-            cp_async16(dv + swz(r, cchunk), Vh + o);
-        }
-    };
-    load_idx(0);
-    issue_tile(0);
-    cp_async_commit();
-    if (ntiles > 1)
-        load_idx(1);
-
-    float o_acc[16][4];
-#pragma unroll
-    for (int n = 0; n < 16; ++n)
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-            o_acc[n][q] = 0.f;
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-    uint32_t qf[8][4];
-    const float sl2 = a.scale * 1.4426950408889634f;
-
-    for (int t = 0; t < ntiles; ++t) {
-        const int stage = t & 1;
-        if (t + 1 < ntiles) {
-            issue_tile(stage ^ 1);
+            for (int i = 0; i < BN / 8; ++i) {
+                int r = crow + 8 * i;
+                const int64_t o = (int64_t)kidx[i] * a.sn + cchunk * 8;
+                cp_async16(dk + sw128(r, cchunk & 7), Kh + o);
+                cp_async16(dv + sw128(r, cchunk & 7), Vh + o);
+            }
+        };
+        // LA tiles are in flight ahead of the one being handed over; tile t is handed over before
+        // the slot for tile t + LA is waited for (that slot is freed by work that needs tile t)
+        constexpr int LA = STAGES - 1;
+        for (int i = 0; i < LA && i < ntiles; ++i) {
+            load_idx(i);
+            issue_tile(i % STAGES);
             cp_async_commit();
-            if (t + 2 < ntiles)
-                load_idx(t + 2);
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
         }
-        __syncthreads();
-        if (t == 0) {
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-                ldsm_x4(smem_u32(sQ) + swz(warp * 16 + (lane & 15), ks * 2 + (lane >> 4)), qf[ks][0], qf[ks][1],
-                        qf[ks][2], qf[ks][3]);
-        }
-        const uint32_t kb = smem_u32(sK) + stage * TILE_BYTES, vb = smem_u32(sV) + stage * TILE_BYTES;
-
-        // S = Q K^T
-        float s[8][4];
-#pragma unroll
-        for (int n = 0; n < 8; ++n)
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                s[n][q] = 0.f;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-#pragma unroll
-            for (int np = 0; np < 4; ++np) {
-                uint32_t b0, b1, b2, b3;
-                int key = np * 16 + (lane & 7) + ((lane >> 4) << 3);
-                int chunk = ks * 2 + ((lane >> 3) & 1);
-                ldsm_x4(kb + swz(key, chunk), b0, b1, b2, b3);
-                mma_bf16(s[2 * np], qf[ks], b0, b1);
-                mma_bf16(s[2 * np + 1], qf[ks], b2, b3);
+        bool alive = true;
+        for (int t = 0; t < ntiles && alive; ++t) {
+            const int newer = min(LA - 1, ntiles - 1 - t);
+            if (newer <= 0)
+                cp_async_wait<0>();
+            else if (newer == 1)
+                cp_async_wait<1>();
+            else
+                cp_async_wait<2>();
+            fence_proxy_async();
+            if (t == 0)
+                mbar_arrive(&bars.q_full);
+            mbar_arrive(&bars.kv_full[t % STAGES]);
+            const int nt = t + LA;
+            if (nt < ntiles) {
+                load_idx(nt);
+                if (nt >= STAGES)
+                    alive = wait(&bars.kv_empty[nt % STAGES], (uint32_t)((nt / STAGES - 1) & 1), abort_flag);
+                if (!alive)
+                    break;
+                issue_tile(nt % STAGES);
+                cp_async_commit();
             }
         }
-        // mask keys past the end of the list (last tile only)
-        const int kvalid = nkeys - t * BN;
-        if (kvalid < BN) {
+        cp_async_wait<0>();
+    } else if (warp == 4) {
+        // ===================== MMA issue: one thread =====================
+        if (lane == 0) {
+            const uint32_t idesc_s = idesc_bf16(BM, BN, false, false);
+            const uint32_t idesc_o = idesc_bf16(BM, kHeadDim, false, true);  // V is read MN-major
+            const uint32_t qb = smem_u32(sQ), pb = smem_u32(sP);
+            auto issue_s = [&](int t) {
+                const uint32_t kb = smem_u32(sKV) + (t % STAGES) * 2 * TILE;
+                const uint32_t d = tmem + ((t & 1) ? COL_S1 : COL_S0);
 #pragma unroll
-            for (int n = 0; n < 8; ++n) {
-                int col = n * 8 + (lane & 3) * 2;
-                if (col >= kvalid)
-                    s[n][0] = s[n][2] = -INFINITY;
-                if (col + 1 >= kvalid)
-                    s[n][1] = s[n][3] = -INFINITY;
+                for (int ks = 0; ks < 8; ++ks) {
+                    uint64_t da = smem_desc_sw128(qb + (ks >> 2) * HALF + (ks & 3) * 32);
+                    uint64_t db = smem_desc_sw128(kb + (ks >> 2) * HALF + (ks & 3) * 32);
+                    mma_ss(d, da, db, idesc_s, ks > 0);
+                }
+                mma_commit(&bars.s_full[t & 1]);
+            };
+            bool alive = wait(&bars.q_full, 0, abort_flag) && wait(&bars.kv_full[0], 0, abort_flag);
+            if (alive) {
+                tc_fence_after();
+                issue_s(0);
+            }
+            for (int t = 0; t < ntiles && alive; ++t) {
+                if (t + 1 < ntiles) {
+                    alive = wait(&bars.kv_full[(t + 1) % STAGES], (uint32_t)(((t + 1) / STAGES) & 1), abort_flag);
+                    if (alive && t + 1 >= 2)
+                        alive = wait(&bars.s_empty[(t + 1) & 1], (uint32_t)(((t + 1) / 2 - 1) & 1), abort_flag);
+                    if (!alive)
+                        break;
+                    tc_fence_after();
+                    issue_s(t + 1);
+                }
+                alive = wait(&bars.p_full, (uint32_t)(t & 1), abort_flag);
+                if (!alive)
+                    break;
+                tc_fence_after();
+                const uint32_t vb = smem_u32(sKV) + (t % STAGES) * 2 * TILE + TILE;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    uint64_t da = smem_desc_sw128(pb + (ks >> 2) * HALF + (ks & 3) * 32);
+                    uint64_t db = smem_desc_sw128(vb + ks * 16 * 128, /*lbo=*/HALF, /*sbo=*/1024);
+                    mma_ss(tmem + COL_O, da, db, idesc_o, t > 0 || ks > 0);
+                }
+                mma_commit(&bars.kv_empty[t % STAGES]);
+                mma_commit(&bars.pv_done);
             }
         }
-        // online softmax (rows lane/4 and lane/4 + 8 of the warp's 16)
-        float mx[2] = {-INFINITY, -INFINITY};
+    } else {
+        // ===================== softmax + correction + epilogue: one thread per query row =====================
+        const int r = tid - (PRODUCER_THREADS + 32);  // row = TMEM lane
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        // warps 5..8: (warp & 3) = 1,2,3,0 -> each warp must touch its own lane quarter
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        (void)r;
+        const float sl2 = a.scale * 1.4426950408889634f;
+        float m_run = -INFINITY, l_run = 0.f;
+        bool alive = true;
+        for (int t = 0; t < ntiles && alive; ++t) {
+            alive = wait(&bars.s_full[t & 1], (uint32_t)((t >> 1) & 1), abort_flag);
+            alive = __all_sync(0xffffffffu, alive);
+            if (!alive)
+                break;
+            tc_fence_after();
+            float s[BN];
+            const uint32_t sa = tmem + lane_addr + ((t & 1) ? COL_S1 : COL_S0);
 #pragma unroll
-        for (int n = 0; n < 8; ++n) {
-            mx[0] = fmaxf(mx[0], fmaxf(s[n][0], s[n][1]));
-            mx[1] = fmaxf(mx[1], fmaxf(s[n][2], s[n][3]));
+            for (int c4 = 0; c4 < 4; ++c4) {
+                uint32_t v[32];
+                tmem_ld32(sa + c4 * 32, v);
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    s[c4 * 32 + j] = __uint_as_float(v[j]);
+            }
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(&bars.s_empty[t & 1]);
+            const int kvalid = nkeys - t * BN;
+            float mx = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < BN; ++j) {
+                if (j >= kvalid)
+                    s[j] = -INFINITY;
+                mx = fmaxf(mx, s[j]);
+            }
+            const float m_new = fmaxf(m_run, mx * sl2);
+            const float alpha = exp2f(m_run - m_new);
+            m_run = m_new;
+            float rs = 0.f;
+            uint32_t p[BN / 2];
+#pragma unroll
+            for (int j = 0; j < BN; j += 2) {
+                float p0 = exp2f(fmaf(s[j], sl2, -m_new));
+                float p1 = exp2f(fmaf(s[j + 1], sl2, -m_new));
+                rs += p0 + p1;
+                p[j >> 1] = pack_bf16(p0, p1);
+            }
+            l_run = l_run * alpha + rs;
+            // the previous P V must be complete before O is rescaled and P is overwritten
+            if (t > 0) {
+                alive = wait(&bars.pv_done, (uint32_t)((t - 1) & 1), abort_flag);
+                alive = __all_sync(0xffffffffu, alive);
+                if (!alive)
+                    break;
+                tc_fence_after();
+                if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        uint32_t v[32];
+                        tmem_ld32(tmem + lane_addr + COL_O + c4 * 32, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
+                        tmem_st32(tmem + lane_addr + COL_O + c4 * 32, v);
+                    }
+                    tmem_wait_st();
+                }
+            }
+            // P row -> shared memory, K-major (keys), 16 chunks of 8 keys
+#pragma unroll
+            for (int ch = 0; ch < 16; ++ch) {
+                uint4 v = make_uint4(p[ch * 4], p[ch * 4 + 1], p[ch * 4 + 2], p[ch * 4 + 3]);
+                *reinterpret_cast<uint4 *>(sP + (ch >> 3) * HALF + sw128(row, ch & 7)) = v;
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(&bars.p_full);
         }
-        float alpha[2], msc[2];
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-            mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 1));
-            mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 2));
-            float mnew = fmaxf(m_run[hh], mx[hh] * sl2);
-            alpha[hh] = exp2f(m_run[hh] - mnew);
-            m_run[hh] = mnew;
-            msc[hh] = mnew;
+        if (alive) {
+            alive = wait(&bars.pv_done, (uint32_t)((ntiles - 1) & 1), abort_flag);
+            alive = __all_sync(0xffffffffu, alive);
         }
-        float rs[2] = {0.f, 0.f};
-        uint32_t pf[4][4];
+        if (alive) {
+            tc_fence_after();
+            const float inv = 1.f / l_run;
+            const bool ok = row < nrows;
+            const int tok = ok ? (rowlist ? rowlist[row] : row0 + row) : 0;
+            bf16 *orow = Oh + (int64_t)tok * a.sn;
 #pragma unroll
-        for (int n = 0; n < 8; ++n) {
-            float p0 = exp2f(fmaf(s[n][0], sl2, -msc[0]));
-            float p1 = exp2f(fmaf(s[n][1], sl2, -msc[0]));
-            float p2 = exp2f(fmaf(s[n][2], sl2, -msc[1]));
-            float p3 = exp2f(fmaf(s[n][3], sl2, -msc[1]));
-            rs[0] += p0 + p1;
-            rs[1] += p2 + p3;
-            pf[n >> 1][(n & 1) * 2] = pack_bf16(p0, p1);
-            pf[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
-        }
+            for (int c4 = 0; c4 < 4; ++c4) {
+                uint32_t v[32];
+                tmem_ld32(tmem + lane_addr + COL_O + c4 * 32, v);
+                tmem_wait_ld();
+                if (ok) {
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh)
-            l_run[hh] = l_run[hh] * alpha[hh] + rs[hh];
-#pragma unroll
-        for (int n = 0; n < 16; ++n) {
-            o_acc[n][0] *= alpha[0];
-            o_acc[n][1] *= alpha[0];
-            o_acc[n][2] *= alpha[1];
-            o_acc[n][3] *= alpha[1];
-        }
-        // O += P V
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-#pragma unroll
-            for (int dp = 0; dp < 8; ++dp) {
-                uint32_t b0, b1, b2, b3;
-                int key = kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
-                int chunk = dp * 2 + (lane >> 4);
-                ldsm_x4_t(vb + swz(key, chunk), b0, b1, b2, b3);
-                mma_bf16(o_acc[2 * dp], pf[kk], b0, b1);
-                mma_bf16(o_acc[2 * dp + 1], pf[kk], b2, b3);
+                    for (int j = 0; j < 32; j += 8) {
+                        uint4 o;
+                        o.x = pack_bf16(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv);
+                        o.y = pack_bf16(__uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv);
+                        o.z = pack_bf16(__uint_as_float(v[j + 4]) * inv, __uint_as_float(v[j + 5]) * inv);
+                        o.w = pack_bf16(__uint_as_float(v[j + 6]) * inv, __uint_as_float(v[j + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(orow + c4 * 32 + j) = o;
+                    }
+                }
             }
         }
-        __syncthreads();
     }
 
-    // normalise, stage the tile in shared memory, write whole rows
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-        float l = l_run[hh];
-        l += __shfl_xor_sync(0xffffffffu, l, 1);
-        l += __shfl_xor_sync(0xffffffffu, l, 2);
-        l_run[hh] = 1.f / l;
-    }
-    {
-        const int r0 = warp * 16 + (lane >> 2);
-#pragma unroll
-        for (int n = 0; n < 16; ++n) {
-            // n-tile n covers channels 8n..8n+7 = chunk n; this thread holds 2 of them
-            uint32_t lo = pack_bf16(o_acc[n][0] * l_run[0], o_acc[n][1] * l_run[0]);
-            uint32_t hi = pack_bf16(o_acc[n][2] * l_run[1], o_acc[n][3] * l_run[1]);
-            *reinterpret_cast<uint32_t *>(sQ + swz(r0, n) + (lane & 3) * 4) = lo;
-            *reinterpret_cast<uint32_t *>(sQ + swz(r0 + 8, n) + (lane & 3) * 4) = hi;
-        }
-    }
+    tc_fence_before();
     __syncthreads();
-#pragma unroll
-    for (int i = 0; i < BM / 8; ++i) {
-        int r = crow + 8 * i;
-        if (r < nrows) {
-            int tok = rowlist ? rowlist[r] : row0 + r;
-            uint4 v = *reinterpret_cast<const uint4 *>(sQ + swz(r, cchunk));
-            *reinterpret_cast<uint4 *>(Oh + (int64_t)tok * a.sn + cchunk * 8) = v;
-        }
-    }
+    if (warp == 4)
+        tmem_dealloc(tmem, TMEM_COLS);
+    if (tid == 0 && s_abort)
+        atomicCAS(status_out + ST_CODE, 0, (int)SCOPE_ERR_TIMEOUT);
 }
 
 }  // namespace
 
 void launch_attn(const AttnArgs &a, cudaStream_t st)
 {
-    const int smem = BM * ROW_BYTES + 4 * TILE_BYTES;
-    cudaFuncSetAttribute(sparse_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaFuncSetAttribute(sparse_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     dim3 grid(a.max_tiles_per_head, a.B * a.H);
-    sparse_attn_kernel<<<grid, NT, smem, st>>>(a);
+    sparse_attn_kernel<<<grid, NT, SMEM_BYTES, st>>>(a, const_cast<int32_t *>(a.status));
     count_launch();
 }
 
