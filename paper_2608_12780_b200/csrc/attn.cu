@@ -44,20 +44,31 @@ struct Barriers {
     uint64_t pv_done;
 };
 
-// bounded wait that also gives up when another role has already failed
+// bounded wait (about a second of SM clock) that also gives up when another role has already failed
 __device__ __forceinline__ bool wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
-    for (uint32_t i = 0; i < 4000000u; ++i) {
+    if (mbar_try_wait(bar, parity))
+        return true;
+    const long long t0 = clock64();
+    for (uint32_t i = 1;; ++i) {
         if (mbar_try_wait(bar, parity))
             return true;
-        if (i > 32) {
-            __nanosleep(40);
-            if ((i & 255u) == 0 && *abort_flag)
+        if ((i & 1023u) == 0) {
+            if (*abort_flag)
                 return false;
+            if (clock64() - t0 > 2000000000ll)
+                break;
         }
     }
     *abort_flag = 1;
     return false;
+}
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
@@ -285,26 +296,47 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
             tc_fence_before();
             mbar_arrive(&bars.s_empty[t & 1]);
             const int kvalid = nkeys - t * BN;
-            float mx = -INFINITY;
+            if (kvalid < BN) {  // last tile of the list: keys past its end carry no weight
 #pragma unroll
-            for (int j = 0; j < BN; ++j) {
-                if (j >= kvalid)
-                    s[j] = -INFINITY;
-                mx = fmaxf(mx, s[j]);
+                for (int j = 0; j < BN; ++j)
+                    if (j >= kvalid)
+                        s[j] = -INFINITY;
             }
-            const float m_new = fmaxf(m_run, mx * sl2);
-            const float alpha = exp2f(m_run - m_new);
-            m_run = m_new;
-            float rs = 0.f;
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int j = 0; j < BN; j += 4) {
+                mx4[0] = fmaxf(mx4[0], s[j]);
+                mx4[1] = fmaxf(mx4[1], s[j + 1]);
+                mx4[2] = fmaxf(mx4[2], s[j + 2]);
+                mx4[3] = fmaxf(mx4[3], s[j + 3]);
+            }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            // The reference maximum only moves when the row maximum has grown by more than 2^8: until
+            // then the weights are at most 2^8, which fp32 sums and bf16 P hold without loss, and the
+            // accumulator in tensor memory needs no rescaling.  Exact in exact arithmetic either way.
+            const float m_cand = mx * sl2;
+            float alpha = 1.f;
+            if (m_cand > m_run + 8.f) {
+                alpha = ex2(m_run - m_cand);
+                m_run = m_cand;
+            }
+            const float neg_m = -m_run;
+            float rs4[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t p[BN / 2];
 #pragma unroll
-            for (int j = 0; j < BN; j += 2) {
-                float p0 = exp2f(fmaf(s[j], sl2, -m_new));
-                float p1 = exp2f(fmaf(s[j + 1], sl2, -m_new));
-                rs += p0 + p1;
+            for (int j = 0; j < BN; j += 4) {
+                float p0 = ex2(fmaf(s[j], sl2, neg_m));
+                float p1 = ex2(fmaf(s[j + 1], sl2, neg_m));
+                float p2 = ex2(fmaf(s[j + 2], sl2, neg_m));
+                float p3 = ex2(fmaf(s[j + 3], sl2, neg_m));
+                rs4[0] += p0;
+                rs4[1] += p1;
+                rs4[2] += p2;
+                rs4[3] += p3;
                 p[j >> 1] = pack_bf16(p0, p1);
+                p[(j >> 1) + 1] = pack_bf16(p2, p3);
             }
-            l_run = l_run * alpha + rs;
+            l_run = l_run * alpha + ((rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
             // the previous P V must be complete before O is rescaled and P is overwritten
             if (t > 0) {
                 alive = wait(&bars.pv_done, (uint32_t)((t - 1) & 1), abort_flag);

@@ -69,17 +69,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after `limit` polls and returns false (the caller records a time-out
-// and leaves; nothing in this library spins forever).
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint32_t limit = 20000000u)
+// Bounded wait: gives up after about a second of SM clock and returns false (the caller records
+// a time-out and leaves; nothing in this library spins forever).
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
 {
-    for (uint32_t i = 0; i < limit; ++i) {
+    if (mbar_try_wait(bar, parity))
+        return true;
+    const long long t0 = clock64();
+    for (uint32_t i = 1;; ++i) {
         if (mbar_try_wait(bar, parity))
             return true;
-        if (i > 64)
-            __nanosleep(32);
+        if ((i & 1023u) == 0 && clock64() - t0 > 2000000000ll)
+            return false;
     }
-    return false;
 }
 
 // ---- tensor memory ------------------------------------------------------------------------------
