@@ -27,10 +27,11 @@ constexpr int BM = kAttnTileRows;  // 128 query rows per block = MMA M
 constexpr int BN = 128;            // keys per tile
 constexpr int HALF = BM * 128;     // bytes of one 64-column half of a 128-row swizzled tile
 constexpr int TILE = 2 * HALF;     // 32 KB: a [128][128] bf16 tile
-constexpr int STAGES = 2;
+constexpr bool P_IN_TMEM = true;   // P as the A operand straight from tensor memory (aliases its S buffer)
+constexpr int STAGES = P_IN_TMEM ? 3 : 2;
 constexpr int PRODUCER_THREADS = 128, SOFTMAX_THREADS = 128;
 constexpr int NT = PRODUCER_THREADS + 32 + SOFTMAX_THREADS;  // 288
-constexpr int SMEM_BYTES = 1024 + TILE /*Q*/ + STAGES * 2 * TILE /*K,V*/ + TILE /*P*/;
+constexpr int SMEM_BYTES = 1024 + TILE /*Q*/ + STAGES * 2 * TILE /*K,V*/ + (P_IN_TMEM ? 0 : TILE) /*P*/;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O = 256;
 
@@ -257,9 +258,14 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
                 const uint32_t vb = smem_u32(sKV) + (t % STAGES) * 2 * TILE + TILE;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    uint64_t da = smem_desc_sw128(pb + (ks >> 2) * HALF + (ks & 3) * 32);
                     uint64_t db = smem_desc_sw128(vb + ks * 16 * 128, /*lbo=*/HALF, /*sbo=*/1024);
-                    mma_ss(tmem + COL_O, da, db, idesc_o, t > 0 || ks > 0);
+                    if (P_IN_TMEM) {
+                        // 16 keys of bf16 P = 8 packed 32-bit columns of the S buffer
+                        mma_ts(tmem + COL_O, tmem + ((t & 1) ? COL_S1 : COL_S0) + ks * 8, db, idesc_o, t > 0 || ks > 0);
+                    } else {
+                        uint64_t da = smem_desc_sw128(pb + (ks >> 2) * HALF + (ks & 3) * 32);
+                        mma_ss(tmem + COL_O, da, db, idesc_o, t > 0 || ks > 0);
+                    }
                 }
                 mma_commit(&bars.kv_empty[t % STAGES]);
                 mma_commit(&bars.pv_done);
@@ -358,13 +364,26 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
                     tmem_wait_st();
                 }
             }
-            // P row -> shared memory, K-major (keys), 16 chunks of 8 keys
+            if (P_IN_TMEM) {
+                // P row (bf16 pairs) over the first 64 columns of its own S buffer
+                uint32_t lo[32], hi[32];
 #pragma unroll
-            for (int ch = 0; ch < 16; ++ch) {
-                uint4 v = make_uint4(p[ch * 4], p[ch * 4 + 1], p[ch * 4 + 2], p[ch * 4 + 3]);
-                *reinterpret_cast<uint4 *>(sP + (ch >> 3) * HALF + sw128(row, ch & 7)) = v;
+                for (int j = 0; j < 32; ++j) {
+                    lo[j] = p[j];
+                    hi[j] = p[32 + j];
+                }
+                tmem_st32(sa, lo);
+                tmem_st32(sa + 32, hi);
+                tmem_wait_st();
+            } else {
+                // P row -> shared memory, K-major (keys), 16 chunks of 8 keys
+#pragma unroll
+                for (int ch = 0; ch < 16; ++ch) {
+                    uint4 v = make_uint4(p[ch * 4], p[ch * 4 + 1], p[ch * 4 + 2], p[ch * 4 + 3]);
+                    *reinterpret_cast<uint4 *>(sP + (ch >> 3) * HALF + sw128(row, ch & 7)) = v;
+                }
+                fence_proxy_async();
             }
-            fence_proxy_async();
             tc_fence_before();
             mbar_arrive(&bars.p_full);
         }
