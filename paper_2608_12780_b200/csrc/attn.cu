@@ -6,12 +6,13 @@
 // queries of one cluster (gathered through the query permutation) and streams the cluster's key
 // list in tiles of 128 gathered K and V rows:
 //   * 4 producer warps gather K/V rows with 16-byte cp.async into 128-byte-swizzled shared
-//     memory, two tiles in flight;
+//     memory, three stages;
 //   * 1 MMA warp (one thread) issues S = Q K^T (accumulator in tensor memory, double buffered)
 //     and O += P V (accumulator in tensor memory);
-//   * 4 softmax warps, one thread per query row (= TMEM lane): read S, keep the running row
-//     maximum and row sum in registers, rescale O in tensor memory when the maximum grows, write
-//     P (bf16) as the A operand of the second MMA.
+//   * 8 softmax warps, two threads per query row (= TMEM lane, 64 keys each): read S, keep the
+//     running row maximum and row sum in registers, rescale O in tensor memory when the maximum
+//     has grown by more than 2^8, write P (bf16) over their S buffer in tensor memory, from where
+//     it is the A operand of the second MMA.
 // Roles synchronise through mbarriers only; every wait is bounded and a time-out ends the block
 // with an error status instead of hanging.
 #include "scope_internal.cuh"
@@ -27,11 +28,11 @@ constexpr int BM = kAttnTileRows;  // 128 query rows per block = MMA M
 constexpr int BN = 128;            // keys per tile
 constexpr int HALF = BM * 128;     // bytes of one 64-column half of a 128-row swizzled tile
 constexpr int TILE = 2 * HALF;     // 32 KB: a [128][128] bf16 tile
-constexpr bool P_IN_TMEM = true;   // P as the A operand straight from tensor memory (aliases its S buffer)
-constexpr int STAGES = P_IN_TMEM ? 3 : 2;
-constexpr int PRODUCER_THREADS = 128, SOFTMAX_THREADS = 128;
-constexpr int NT = PRODUCER_THREADS + 32 + SOFTMAX_THREADS;  // 288
-constexpr int SMEM_BYTES = 1024 + TILE /*Q*/ + STAGES * 2 * TILE /*K,V*/ + (P_IN_TMEM ? 0 : TILE) /*P*/;
+constexpr int STAGES = 3;
+constexpr int PRODUCER_THREADS = 128, SOFTMAX_THREADS = 256;
+constexpr int NT = PRODUCER_THREADS + 32 + SOFTMAX_THREADS;  // 416
+constexpr int TILES_BYTES = TILE /*Q*/ + STAGES * 2 * TILE /*K,V*/;
+constexpr int SMEM_BYTES = TILES_BYTES + 2048 /*row exchange*/ + 256 /*barriers*/;  // all of an SM's 227 KB
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O = 256;
 
@@ -40,9 +41,9 @@ struct Barriers {
     uint64_t kv_full[STAGES];
     uint64_t kv_empty[STAGES];
     uint64_t s_full[2];
-    uint64_t s_empty[2];
     uint64_t p_full;
     uint64_t pv_done;
+    uint64_t x_full;  // exchange between the two threads of a row
 };
 
 // bounded wait (about a second of SM clock) that also gives up when another role has already failed
@@ -80,17 +81,23 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 
 __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t *status_out)
 {
-    extern __shared__ unsigned char smem_dyn[];
-    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    // the whole shared memory of the SM, laid out by hand: swizzled tiles first (1024-byte aligned)
+    extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *sQ = smem;
     unsigned char *sKV = sQ + TILE;                 // stage s: K at sKV + s*2*TILE, V right after
-    unsigned char *sP = sKV + STAGES * 2 * TILE;
-    __shared__ Barriers bars;
-    __shared__ uint32_t s_tmem_base;
-    __shared__ int s_abort;
+    float (*s_rowmax)[2][BM] = reinterpret_cast<float (*)[2][BM]>(smem + TILES_BYTES);  // [2][2][BM]
+    Barriers &bars = *reinterpret_cast<Barriers *>(smem + TILES_BYTES + 2048);
+    uint32_t &s_tmem_base = *reinterpret_cast<uint32_t *>(smem + TILES_BYTES + 2048 + 128);
+    int &s_abort = *reinterpret_cast<int *>(smem + TILES_BYTES + 2048 + 132);
+    static_assert(sizeof(Barriers) <= 128, "barrier block");
 
     if (!a.dense && a.status[ST_CODE] != 0)
         return;
+    if (smem_u32(smem) & 1023u) {  // the swizzled layouts need it; never seen, but never assumed
+        if (threadIdx.x == 0)
+            atomicCAS(status_out + ST_CODE, 0, (int)SCOPE_ERR_CUDA);
+        return;
+    }
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.y;
     const int b = bh / a.H, h = bh % a.H;
@@ -141,10 +148,10 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(&bars.s_full[s], 1);
-            mbar_init(&bars.s_empty[s], SOFTMAX_THREADS);
         }
         mbar_init(&bars.p_full, SOFTMAX_THREADS);
         mbar_init(&bars.pv_done, 1);
+        mbar_init(&bars.x_full, SOFTMAX_THREADS);
         mbar_fence_init();
     }
     if (warp == 4) {
@@ -224,7 +231,7 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
         if (lane == 0) {
             const uint32_t idesc_s = idesc_bf16(BM, BN, false, false);
             const uint32_t idesc_o = idesc_bf16(BM, kHeadDim, false, true);  // V is read MN-major
-            const uint32_t qb = smem_u32(sQ), pb = smem_u32(sP);
+            const uint32_t qb = smem_u32(sQ);
             auto issue_s = [&](int t) {
                 const uint32_t kb = smem_u32(sKV) + (t % STAGES) * 2 * TILE;
                 const uint32_t d = tmem + ((t & 1) ? COL_S1 : COL_S0);
@@ -244,8 +251,6 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
             for (int t = 0; t < ntiles && alive; ++t) {
                 if (t + 1 < ntiles) {
                     alive = wait(&bars.kv_full[(t + 1) % STAGES], (uint32_t)(((t + 1) / STAGES) & 1), abort_flag);
-                    if (alive && t + 1 >= 2)
-                        alive = wait(&bars.s_empty[(t + 1) & 1], (uint32_t)(((t + 1) / 2 - 1) & 1), abort_flag);
                     if (!alive)
                         break;
                     tc_fence_after();
@@ -259,26 +264,21 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     uint64_t db = smem_desc_sw128(vb + ks * 16 * 128, /*lbo=*/HALF, /*sbo=*/1024);
-                    if (P_IN_TMEM) {
-                        // 16 keys of bf16 P = 8 packed 32-bit columns of the S buffer
-                        mma_ts(tmem + COL_O, tmem + ((t & 1) ? COL_S1 : COL_S0) + ks * 8, db, idesc_o, t > 0 || ks > 0);
-                    } else {
-                        uint64_t da = smem_desc_sw128(pb + (ks >> 2) * HALF + (ks & 3) * 32);
-                        mma_ss(tmem + COL_O, da, db, idesc_o, t > 0 || ks > 0);
-                    }
+                    // A = P straight from tensor memory: 16 keys of bf16 = 8 packed 32-bit columns of the S buffer
+                    mma_ts(tmem + COL_O, tmem + ((t & 1) ? COL_S1 : COL_S0) + ks * 8, db, idesc_o, t > 0 || ks > 0);
                 }
                 mma_commit(&bars.kv_empty[t % STAGES]);
                 mma_commit(&bars.pv_done);
             }
         }
     } else {
-        // ===================== softmax + correction + epilogue: one thread per query row =====================
-        const int r = tid - (PRODUCER_THREADS + 32);  // row = TMEM lane
+        // ============ softmax + correction + epilogue: two threads per query row (64 keys each) ============
+        // warps 5..8 take keys 0..63 of the tile, warps 9..12 keys 64..127; a warp may only touch the
+        // TMEM lane quarter (warp & 3), which for both sets runs through 1,2,3,0
+        const int half = (warp - 5) >> 2;
+        const int row = (warp & 3) * 32 + lane;  // query row = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        // warps 5..8: (warp & 3) = 1,2,3,0 -> each warp must touch its own lane quarter
-        const int q = warp & 3;
-        const int row = q * 32 + lane;
-        (void)r;
+        constexpr int HN = BN / 2;               // keys per thread
         const float sl2 = a.scale * 1.4426950408889634f;
         float m_run = -INFINITY, l_run = 0.f;
         bool alive = true;
@@ -288,35 +288,42 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
             if (!alive)
                 break;
             tc_fence_after();
-            float s[BN];
+            float s[HN];
             const uint32_t sa = tmem + lane_addr + ((t & 1) ? COL_S1 : COL_S0);
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
+            for (int c2 = 0; c2 < HN / 32; ++c2) {
                 uint32_t v[32];
-                tmem_ld32(sa + c4 * 32, v);
+                tmem_ld32(sa + half * HN + c2 * 32, v);
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
-                    s[c4 * 32 + j] = __uint_as_float(v[j]);
+                    s[c2 * 32 + j] = __uint_as_float(v[j]);
             }
             tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(&bars.s_empty[t & 1]);
-            const int kvalid = nkeys - t * BN;
-            if (kvalid < BN) {  // last tile of the list: keys past its end carry no weight
+            const int kvalid = nkeys - t * BN - half * HN;
+            if (kvalid < HN) {  // last tile of the list: keys past its end carry no weight
 #pragma unroll
-                for (int j = 0; j < BN; ++j)
+                for (int j = 0; j < HN; ++j)
                     if (j >= kvalid)
                         s[j] = -INFINITY;
             }
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int j = 0; j < BN; j += 4) {
+            for (int j = 0; j < HN; j += 4) {
                 mx4[0] = fmaxf(mx4[0], s[j]);
                 mx4[1] = fmaxf(mx4[1], s[j + 1]);
                 mx4[2] = fmaxf(mx4[2], s[j + 2]);
                 mx4[3] = fmaxf(mx4[3], s[j + 3]);
             }
-            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            // the two halves of a row agree on one maximum (the exchange also orders every read of
+            // S before any write of P into the same columns)
+            s_rowmax[t & 1][half][row] = mx;
+            mbar_arrive(&bars.x_full);
+            alive = wait(&bars.x_full, (uint32_t)(t & 1), abort_flag);
+            alive = __all_sync(0xffffffffu, alive);
+            if (!alive)
+                break;
+            mx = fmaxf(mx, s_rowmax[t & 1][half ^ 1][row]);
             // The reference maximum only moves when the row maximum has grown by more than 2^8: until
             // then the weights are at most 2^8, which fp32 sums and bf16 P hold without loss, and the
             // accumulator in tensor memory needs no rescaling.  Exact in exact arithmetic either way.
@@ -328,9 +335,9 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
             }
             const float neg_m = -m_run;
             float rs4[4] = {0.f, 0.f, 0.f, 0.f};
-            uint32_t p[BN / 2];
+            uint32_t p[HN / 2];
 #pragma unroll
-            for (int j = 0; j < BN; j += 4) {
+            for (int j = 0; j < HN; j += 4) {
                 float p0 = ex2(fmaf(s[j], sl2, neg_m));
                 float p1 = ex2(fmaf(s[j + 1], sl2, neg_m));
                 float p2 = ex2(fmaf(s[j + 2], sl2, neg_m));
@@ -343,49 +350,39 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
                 p[(j >> 1) + 1] = pack_bf16(p2, p3);
             }
             l_run = l_run * alpha + ((rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
-            // the previous P V must be complete before O is rescaled and P is overwritten
-            if (t > 0) {
+            // O is rescaled only when some row of this warp moved its reference maximum, and only
+            // then must the previous P V be complete (P itself lives in its own S buffer)
+            const bool rescale = __any_sync(0xffffffffu, alpha != 1.f);
+            if (t > 0 && rescale) {
                 alive = wait(&bars.pv_done, (uint32_t)((t - 1) & 1), abort_flag);
                 alive = __all_sync(0xffffffffu, alive);
                 if (!alive)
                     break;
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        uint32_t v[32];
-                        tmem_ld32(tmem + lane_addr + COL_O + c4 * 32, v);
-                        tmem_wait_ld();
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem + lane_addr + COL_O + half * 64 + c2 * 32, v);
+                    tmem_wait_ld();
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
-                        tmem_st32(tmem + lane_addr + COL_O + c4 * 32, v);
-                    }
-                    tmem_wait_st();
+                    for (int j = 0; j < 32; ++j)
+                        v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
+                    tmem_st32(tmem + lane_addr + COL_O + half * 64 + c2 * 32, v);
                 }
-            }
-            if (P_IN_TMEM) {
-                // P row (bf16 pairs) over the first 64 columns of its own S buffer
-                uint32_t lo[32], hi[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    lo[j] = p[j];
-                    hi[j] = p[32 + j];
-                }
-                tmem_st32(sa, lo);
-                tmem_st32(sa + 32, hi);
                 tmem_wait_st();
-            } else {
-                // P row -> shared memory, K-major (keys), 16 chunks of 8 keys
-#pragma unroll
-                for (int ch = 0; ch < 16; ++ch) {
-                    uint4 v = make_uint4(p[ch * 4], p[ch * 4 + 1], p[ch * 4 + 2], p[ch * 4 + 3]);
-                    *reinterpret_cast<uint4 *>(sP + (ch >> 3) * HALF + sw128(row, ch & 7)) = v;
-                }
-                fence_proxy_async();
             }
+            // P row (bf16 pairs): keys 64*half.. of the tile = packed columns 32*half.. of the S buffer
+            tmem_st32(sa + half * (HN / 2), p);
+            tmem_wait_st();
             tc_fence_before();
             mbar_arrive(&bars.p_full);
+        }
+        if (alive) {
+            // row sums of the two halves meet in shared memory
+            s_rowmax[ntiles & 1][half][row] = l_run;
+            mbar_arrive(&bars.x_full);
+            alive = wait(&bars.x_full, (uint32_t)(ntiles & 1), abort_flag);
+            alive = __all_sync(0xffffffffu, alive);
         }
         if (alive) {
             alive = wait(&bars.pv_done, (uint32_t)((ntiles - 1) & 1), abort_flag);
@@ -393,14 +390,14 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
         }
         if (alive) {
             tc_fence_after();
-            const float inv = 1.f / l_run;
+            const float inv = 1.f / (l_run + s_rowmax[ntiles & 1][half ^ 1][row]);
             const bool ok = row < nrows;
             const int tok = ok ? (rowlist ? rowlist[row] : row0 + row) : 0;
-            bf16 *orow = Oh + (int64_t)tok * a.sn;
+            bf16 *orow = Oh + (int64_t)tok * a.sn + half * 64;
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
+            for (int c2 = 0; c2 < 2; ++c2) {
                 uint32_t v[32];
-                tmem_ld32(tmem + lane_addr + COL_O + c4 * 32, v);
+                tmem_ld32(tmem + lane_addr + COL_O + half * 64 + c2 * 32, v);
                 tmem_wait_ld();
                 if (ok) {
 #pragma unroll
@@ -410,7 +407,7 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
                         o.y = pack_bf16(__uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv);
                         o.z = pack_bf16(__uint_as_float(v[j + 4]) * inv, __uint_as_float(v[j + 5]) * inv);
                         o.w = pack_bf16(__uint_as_float(v[j + 6]) * inv, __uint_as_float(v[j + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(orow + c4 * 32 + j) = o;
+                        *reinterpret_cast<uint4 *>(orow + c2 * 32 + j) = o;
                     }
                 }
             }
