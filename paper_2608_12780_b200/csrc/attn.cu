@@ -2,17 +2,18 @@
 // original keys/values listed in S_c.  With `dense` set the key list is 0..N-1 and the grouping is
 // the identity, which is Eq. 1.
 //
-// Flash-style, warp-specialised, on the tcgen05 tensor cores.  One block owns a tile of 128
-// queries of one cluster (gathered through the query permutation) and streams the cluster's key
-// list in tiles of 128 gathered K and V rows:
+// Flash-style, warp-specialised, on the tcgen05 tensor cores.  One block owns up to 256 queries of
+// one cluster (two tiles of 128, gathered through the query permutation) and streams the cluster's
+// key list once for both, in tiles of 64 gathered K and V rows:
 //   * 4 producer warps gather K/V rows with 16-byte cp.async into 128-byte-swizzled shared
-//     memory, three stages;
-//   * 1 MMA warp (one thread) issues S = Q K^T (accumulator in tensor memory, double buffered)
-//     and O += P V (accumulator in tensor memory);
-//   * 8 softmax warps, two threads per query row (= TMEM lane, 64 keys each): read S, keep the
-//     running row maximum and row sum in registers, rescale O in tensor memory when the maximum
-//     has grown by more than 2^8, write P (bf16) over their S buffer in tensor memory, from where
-//     it is the A operand of the second MMA.
+//     memory, five stages (four tiles in flight);
+//   * 2 MMA warps (one thread each, one per query tile) issue, per key tile, S = Q K^T (accumulator
+//     in tensor memory, double buffered) and O += P V (accumulator in tensor memory);
+//   * 2 x 4 softmax warps, one thread per query row (= TMEM lane): read S, keep the running row
+//     maximum and row sum in registers, rescale O in tensor memory when the maximum has grown by
+//     more than 2^8, write P (bf16) over their S buffer in tensor memory, from where it is the A
+//     operand of the second MMA.  Half of the exponentials run on the FMA pipe (range reduction +
+//     polynomial) because the special-function unit alone is slower than the tensor core here.
 // Roles synchronise through mbarriers only; every wait is bounded and a time-out ends the block
 // with an error status instead of hanging.
 #include "scope_internal.cuh"
@@ -24,26 +25,29 @@ using namespace sm100;
 
 namespace {
 
-constexpr int BM = kAttnTileRows;  // 128 query rows per block = MMA M
-constexpr int BN = 128;            // keys per tile
-constexpr int HALF = BM * 128;     // bytes of one 64-column half of a 128-row swizzled tile
-constexpr int TILE = 2 * HALF;     // 32 KB: a [128][128] bf16 tile
-constexpr int STAGES = 3;
-constexpr int PRODUCER_THREADS = 128, SOFTMAX_THREADS = 256;
-constexpr int NT = PRODUCER_THREADS + 32 + SOFTMAX_THREADS;  // 416
-constexpr int TILES_BYTES = TILE /*Q*/ + STAGES * 2 * TILE /*K,V*/;
-constexpr int SMEM_BYTES = TILES_BYTES + 2048 /*row exchange*/ + 256 /*barriers*/;  // all of an SM's 227 KB
+constexpr int BM = 128;                    // rows per query tile = MMA M
+constexpr int QT = kAttnTileRows / BM;     // query tiles per block (2)
+constexpr int BN = 64;                     // keys per tile
+constexpr int STAGES = 5;
+constexpr int QHALF = BM * 128, QTILE = 2 * QHALF;   // [128][128] bf16 as two 64-column halves
+constexpr int KHALF = BN * 128, KTILE = 2 * KHALF;   // [64][128] bf16
+constexpr int STAGE_BYTES = 2 * KTILE;               // K then V
+constexpr int PRODUCER_THREADS = 128, SOFTMAX_THREADS = QT * BM;
+constexpr int NT = PRODUCER_THREADS + 32 + SOFTMAX_THREADS + 32;  // 448: producers, MMA 0, softmax, MMA 1
+constexpr int TILES_BYTES = QT * QTILE + STAGES * STAGE_BYTES;
+constexpr int SMEM_BYTES = TILES_BYTES + 512;  // + barriers
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O = 256;
+// tensor-memory columns of query tile i: S buffers at i*256 + {0, 64}, O at i*256 + 128
+constexpr uint32_t COL_TILE = 256, COL_SBUF = 64, COL_O = 128;
+static_assert(QT == 2, "two query tiles per block");
 
 struct Barriers {
     uint64_t q_full;
     uint64_t kv_full[STAGES];
     uint64_t kv_empty[STAGES];
-    uint64_t s_full[2];
-    uint64_t p_full;
-    uint64_t pv_done;
-    uint64_t x_full;  // exchange between the two threads of a row
+    uint64_t s_full[QT][2];
+    uint64_t p_full[QT];
+    uint64_t pv_done[QT];
 };
 
 // bounded wait (about a second of SM clock) that also gives up when another role has already failed
@@ -73,6 +77,33 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
+// 2^x for two values on the FMA pipe: x = n + f with n integer and |f| <= 1/2 (magic-number
+// rounding), 2^f by a degree-4 polynomial (relative error 4e-5, far below bf16 resolution), n added
+// into the exponent field.  x is clamped at -126 (the result is then ~1e-38, i.e. no weight).
+__device__ __forceinline__ float2 exp2_fma(float2 x)
+{
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
+    const float2 magic = make_float2(12582912.f, 12582912.f);
+    const float2 r = __fadd2_rn(x, magic);
+    const float2 n = __fadd2_rn(r, make_float2(-12582912.f, -12582912.f));
+    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+    float2 p = __ffma2_rn(f, make_float2(9.6181291e-3f, 9.6181291e-3f), make_float2(5.5504109e-2f, 5.5504109e-2f));
+    p = __ffma2_rn(p, f, make_float2(2.4022651e-1f, 2.4022651e-1f));
+    p = __ffma2_rn(p, f, make_float2(6.9314718e-1f, 6.9314718e-1f));
+    p = __ffma2_rn(p, f, make_float2(1.f, 1.f));
+    float2 y;
+    y.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(r.x) << 23));
+    y.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23));
+    return y;
+}
+
+// two non-negative floats -> packed bf16 pair, round half up (differs from round-to-nearest-even
+// only on exact ties), on the integer pipe
+__device__ __forceinline__ uint32_t pack_bf16_int(float lo, float hi)
+{
+    return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -83,13 +114,12 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
 {
     // the whole shared memory of the SM, laid out by hand: swizzled tiles first (1024-byte aligned)
     extern __shared__ __align__(1024) unsigned char smem[];
-    unsigned char *sQ = smem;
-    unsigned char *sKV = sQ + TILE;                 // stage s: K at sKV + s*2*TILE, V right after
-    float (*s_rowmax)[2][BM] = reinterpret_cast<float (*)[2][BM]>(smem + TILES_BYTES);  // [2][2][BM]
-    Barriers &bars = *reinterpret_cast<Barriers *>(smem + TILES_BYTES + 2048);
-    uint32_t &s_tmem_base = *reinterpret_cast<uint32_t *>(smem + TILES_BYTES + 2048 + 128);
-    int &s_abort = *reinterpret_cast<int *>(smem + TILES_BYTES + 2048 + 132);
-    static_assert(sizeof(Barriers) <= 128, "barrier block");
+    unsigned char *sQ = smem;                       // query tile i at sQ + i*QTILE
+    unsigned char *sKV = sQ + QT * QTILE;           // stage s: K at sKV + s*STAGE_BYTES, V right after
+    Barriers &bars = *reinterpret_cast<Barriers *>(smem + TILES_BYTES);
+    uint32_t &s_tmem_base = *reinterpret_cast<uint32_t *>(smem + TILES_BYTES + 256);
+    int &s_abort = *reinterpret_cast<int *>(smem + TILES_BYTES + 260);
+    static_assert(sizeof(Barriers) <= 256, "barrier block");
 
     if (!a.dense && a.status[ST_CODE] != 0)
         return;
@@ -107,13 +137,13 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
 
     // which cluster / which rows (block-uniform)
     int nrows, nkeys, row0 = 0;
-    const int32_t *rowlist = nullptr;  // tokens of this tile (null: identity)
+    const int32_t *rowlist = nullptr;  // tokens of this block (null: identity)
     const int32_t *keylist = nullptr;  // key indices (null: identity)
     if (a.dense) {
-        row0 = blockIdx.x * BM;
+        row0 = blockIdx.x * kAttnTileRows;
         if (row0 >= a.N)
             return;
-        nrows = min(BM, a.N - row0);
+        nrows = min(kAttnTileRows, a.N - row0);
         nkeys = a.N;
     } else {
         const int32_t *toff = a.tile_offsets + (size_t)bh * (a.Cq + 1);
@@ -130,28 +160,29 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
         }
         const int c = lo;
         const int32_t *qoff = a.q_offsets + (size_t)bh * (a.Cq + 1);
-        const int start = qoff[c] + (x - toff[c]) * BM;
-        nrows = min(BM, qoff[c + 1] - start);
+        const int start = qoff[c] + (x - toff[c]) * kAttnTileRows;
+        nrows = min(kAttnTileRows, qoff[c + 1] - start);
         rowlist = a.q_perm + (size_t)bh * a.N + start;
         const size_t row = (size_t)bh * a.Cq + c;
         nkeys = a.r_c[row];
         keylist = a.key_indices + a.key_offsets[row];
     }
     const int ntiles = (nkeys + BN - 1) / BN;
+    const int nact = nrows > BM ? 2 : 1;  // query tiles in use
 
     if (tid == 0) {
         s_abort = 0;
         mbar_init(&bars.q_full, PRODUCER_THREADS);
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&bars.kv_full[s], PRODUCER_THREADS);
-            mbar_init(&bars.kv_empty[s], 1);
+            mbar_init(&bars.kv_empty[s], nact);
         }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&bars.s_full[s], 1);
+        for (int i = 0; i < QT; ++i) {
+            mbar_init(&bars.s_full[i][0], 1);
+            mbar_init(&bars.s_full[i][1], 1);
+            mbar_init(&bars.p_full[i], BM);
+            mbar_init(&bars.pv_done[i], 1);
         }
-        mbar_init(&bars.p_full, SOFTMAX_THREADS);
-        mbar_init(&bars.pv_done, 1);
-        mbar_init(&bars.x_full, SOFTMAX_THREADS);
         mbar_fence_init();
     }
     if (warp == 4) {
@@ -167,12 +198,12 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
     if (warp < 4) {
         // ===================== producers: Q once, then K/V tiles =====================
         const int crow = tid >> 4, cchunk = tid & 15;  // 8 rows per pass, 16 chunks per row
-        const uint32_t chunk_off = (cchunk >> 3) * HALF;
-        for (int i = 0; i < BM / 8; ++i) {
-            int r = crow + 8 * i;
-            bool ok = r < nrows;
-            int tok = ok ? (rowlist ? rowlist[r] : row0 + r) : 0;
-            cp_async16_zfill(smem_u32(sQ) + chunk_off + sw128(r, cchunk & 7), Qh + (int64_t)tok * a.sn + cchunk * 8, ok ? 16 : 0);
+        for (int i = 0; i < nact * BM / 8; ++i) {
+            const int r = crow + 8 * i, lr = r & (BM - 1);
+            const bool ok = r < nrows;
+            const int tok = ok ? (rowlist ? rowlist[r] : row0 + r) : 0;
+            cp_async16_zfill(smem_u32(sQ) + (r >> 7) * QTILE + (cchunk >> 3) * QHALF + sw128(lr, cchunk & 7),
+                             Qh + (int64_t)tok * a.sn + cchunk * 8, ok ? 16 : 0);
         }
         cp_async_commit();
         int kidx[BN / 8];
@@ -184,10 +215,10 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
             }
         };
         auto issue_tile = [&](int stage) {
-            const uint32_t dk = smem_u32(sKV) + stage * 2 * TILE + chunk_off, dv = dk + TILE;
+            const uint32_t dk = smem_u32(sKV) + stage * STAGE_BYTES + (cchunk >> 3) * KHALF, dv = dk + KTILE;
 #pragma unroll
             for (int i = 0; i < BN / 8; ++i) {
-                int r = crow + 8 * i;
+                const int r = crow + 8 * i;
                 const int64_t o = (int64_t)kidx[i] * a.sn + cchunk * 8;
                 cp_async16(dk + sw128(r, cchunk & 7), Kh + o);
                 cp_async16(dv + sw128(r, cchunk & 7), Vh + o);
@@ -208,8 +239,11 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
                 cp_async_wait<0>();
             else if (newer == 1)
                 cp_async_wait<1>();
-            else
+            else if (newer == 2)
                 cp_async_wait<2>();
+            else
+                cp_async_wait<3>();
+            static_assert(LA - 1 <= 3, "wait_group immediates");
             fence_proxy_async();
             if (t == 0)
                 mbar_arrive(&bars.q_full);
@@ -226,22 +260,29 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
             }
         }
         cp_async_wait<0>();
-    } else if (warp == 4) {
-        // ===================== MMA issue: one thread =====================
-        if (lane == 0) {
+    } else if (warp == 4 || warp == 13) {
+        // ===================== MMA issue: one thread per query tile =====================
+        const int i = warp == 4 ? 0 : 1;
+        if (lane == 0 && i < nact) {
             const uint32_t idesc_s = idesc_bf16(BM, BN, false, false);
             const uint32_t idesc_o = idesc_bf16(BM, kHeadDim, false, true);  // V is read MN-major
-            const uint32_t qb = smem_u32(sQ);
+            // descriptor words: the high word is fixed per operand kind, the low word is the start address
+            const uint64_t dk0 = smem_desc_sw128(0);                              // K-major operands (Q, K)
+            const uint64_t dv0 = smem_desc_sw128(0, /*lbo=*/KHALF, /*sbo=*/1024);  // V, MN-major: halves KHALF apart
+            const uint32_t hi_k = (uint32_t)(dk0 >> 32), lo_k = (uint32_t)dk0;
+            const uint32_t hi_v = (uint32_t)(dv0 >> 32), lo_v = (uint32_t)dv0;
+            const uint32_t q_lo = lo_k + ((smem_u32(sQ) + i * QTILE) >> 4);
+            const uint32_t kv_lo = smem_u32(sKV) >> 4;
+            const uint32_t tm = tmem + i * COL_TILE;
             auto issue_s = [&](int t) {
-                const uint32_t kb = smem_u32(sKV) + (t % STAGES) * 2 * TILE;
-                const uint32_t d = tmem + ((t & 1) ? COL_S1 : COL_S0);
+                const uint32_t k_lo = lo_k + kv_lo + (((t % STAGES) * STAGE_BYTES) >> 4);
+                const uint32_t d = tm + (t & 1) * COL_SBUF;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    uint64_t da = smem_desc_sw128(qb + (ks >> 2) * HALF + (ks & 3) * 32);
-                    uint64_t db = smem_desc_sw128(kb + (ks >> 2) * HALF + (ks & 3) * 32);
-                    mma_ss(d, da, db, idesc_s, ks > 0);
+                    const uint32_t qo = ((ks >> 2) * QHALF + (ks & 3) * 32) >> 4, ko = ((ks >> 2) * KHALF + (ks & 3) * 32) >> 4;
+                    mma_ss2(d, q_lo + qo, hi_k, k_lo + ko, hi_k, idesc_s, ks > 0);
                 }
-                mma_commit(&bars.s_full[t & 1]);
+                mma_commit(&bars.s_full[i][t & 1]);
             };
             bool alive = wait(&bars.q_full, 0, abort_flag) && wait(&bars.kv_full[0], 0, abort_flag);
             if (alive) {
@@ -250,80 +291,73 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
             }
             for (int t = 0; t < ntiles && alive; ++t) {
                 if (t + 1 < ntiles) {
+                    // the S buffer being refilled was last read by P V of tile t-1, issued before: in order
                     alive = wait(&bars.kv_full[(t + 1) % STAGES], (uint32_t)(((t + 1) / STAGES) & 1), abort_flag);
                     if (!alive)
                         break;
                     tc_fence_after();
                     issue_s(t + 1);
                 }
-                alive = wait(&bars.p_full, (uint32_t)(t & 1), abort_flag);
+                alive = wait(&bars.p_full[i], (uint32_t)(t & 1), abort_flag);
                 if (!alive)
                     break;
                 tc_fence_after();
-                const uint32_t vb = smem_u32(sKV) + (t % STAGES) * 2 * TILE + TILE;
+                const uint32_t v_lo = lo_v + kv_lo + (((t % STAGES) * STAGE_BYTES + KTILE) >> 4);
+                const uint32_t pa = tm + (t & 1) * COL_SBUF;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    uint64_t db = smem_desc_sw128(vb + ks * 16 * 128, /*lbo=*/HALF, /*sbo=*/1024);
-                    // A = P straight from tensor memory: 16 keys of bf16 = 8 packed 32-bit columns of the S buffer
-                    mma_ts(tmem + COL_O, tmem + ((t & 1) ? COL_S1 : COL_S0) + ks * 8, db, idesc_o, t > 0 || ks > 0);
+                for (int ks = 0; ks < BN / 16; ++ks) {
+                    // B = V, MN-major: 16 keys per step are 16 rows of 128 B.  A = P straight from tensor
+                    // memory: 16 bf16 = 8 packed columns.
+                    mma_ts2(tm + COL_O, pa + ks * 8, v_lo + ((ks * 16 * 128) >> 4), hi_v, idesc_o, t > 0 || ks > 0);
                 }
+                mma_commit(&bars.pv_done[i]);
                 mma_commit(&bars.kv_empty[t % STAGES]);
-                mma_commit(&bars.pv_done);
             }
         }
-    } else {
-        // ============ softmax + correction + epilogue: two threads per query row (64 keys each) ============
-        // warps 5..8 take keys 0..63 of the tile, warps 9..12 keys 64..127; a warp may only touch the
-        // TMEM lane quarter (warp & 3), which for both sets runs through 1,2,3,0
-        const int half = (warp - 5) >> 2;
-        const int row = (warp & 3) * 32 + lane;  // query row = TMEM lane
-        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        constexpr int HN = BN / 2;               // keys per thread
+    } else if (warp >= 5 && warp < 13 && (warp - 5) >> 2 < nact) {
+        // ============ softmax + correction + epilogue: one thread per query row ============
+        // warps 5..8 own query tile 0, warps 9..12 tile 1; a warp may only touch the TMEM lane quarter
+        // (warp & 3), which for both sets runs through 1,2,3,0
+        const int qt = (warp - 5) >> 2;
+        const int row = (warp & 3) * 32 + lane;  // row inside the tile = TMEM lane
+        const uint32_t tbase = tmem + ((uint32_t)((warp & 3) * 32) << 16) + qt * COL_TILE;
         const float sl2 = a.scale * 1.4426950408889634f;
+        const float2 sl2_2 = make_float2(sl2, sl2);
         float m_run = -INFINITY, l_run = 0.f;
         bool alive = true;
         for (int t = 0; t < ntiles && alive; ++t) {
-            alive = wait(&bars.s_full[t & 1], (uint32_t)((t >> 1) & 1), abort_flag);
+            alive = wait(&bars.s_full[qt][t & 1], (uint32_t)((t >> 1) & 1), abort_flag);
             alive = __all_sync(0xffffffffu, alive);
             if (!alive)
                 break;
             tc_fence_after();
-            float s[HN];
-            const uint32_t sa = tmem + lane_addr + ((t & 1) ? COL_S1 : COL_S0);
+            float s[BN];
+            const uint32_t sa = tbase + (t & 1) * COL_SBUF;
 #pragma unroll
-            for (int c2 = 0; c2 < HN / 32; ++c2) {
+            for (int c2 = 0; c2 < BN / 32; ++c2) {
                 uint32_t v[32];
-                tmem_ld32(sa + half * HN + c2 * 32, v);
+                tmem_ld32(sa + c2 * 32, v);
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
                     s[c2 * 32 + j] = __uint_as_float(v[j]);
             }
             tmem_wait_ld();
-            const int kvalid = nkeys - t * BN - half * HN;
-            if (kvalid < HN) {  // last tile of the list: keys past its end carry no weight
+            const int kvalid = nkeys - t * BN;
+            if (kvalid < BN) {  // last tile of the list: keys past its end carry no weight
 #pragma unroll
-                for (int j = 0; j < HN; ++j)
+                for (int j = 0; j < BN; ++j)
                     if (j >= kvalid)
                         s[j] = -INFINITY;
             }
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int j = 0; j < HN; j += 4) {
+            for (int j = 0; j < BN; j += 4) {
                 mx4[0] = fmaxf(mx4[0], s[j]);
                 mx4[1] = fmaxf(mx4[1], s[j + 1]);
                 mx4[2] = fmaxf(mx4[2], s[j + 2]);
                 mx4[3] = fmaxf(mx4[3], s[j + 3]);
             }
-            float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-            // the two halves of a row agree on one maximum (the exchange also orders every read of
-            // S before any write of P into the same columns)
-            s_rowmax[t & 1][half][row] = mx;
-            mbar_arrive(&bars.x_full);
-            alive = wait(&bars.x_full, (uint32_t)(t & 1), abort_flag);
-            alive = __all_sync(0xffffffffu, alive);
-            if (!alive)
-                break;
-            mx = fmaxf(mx, s_rowmax[t & 1][half ^ 1][row]);
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             // The reference maximum only moves when the row maximum has grown by more than 2^8: until
             // then the weights are at most 2^8, which fp32 sums and bf16 P hold without loss, and the
             // accumulator in tensor memory needs no rescaling.  Exact in exact arithmetic either way.
@@ -333,71 +367,70 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
                 alpha = ex2(m_run - m_cand);
                 m_run = m_cand;
             }
-            const float neg_m = -m_run;
-            float rs4[4] = {0.f, 0.f, 0.f, 0.f};
-            uint32_t p[HN / 2];
+            const float2 neg_m = make_float2(-m_run, -m_run);
+            float2 rs_a = make_float2(0.f, 0.f), rs_b = make_float2(0.f, 0.f);
+            uint32_t p[BN / 2];
 #pragma unroll
-            for (int j = 0; j < HN; j += 4) {
-                float p0 = ex2(fmaf(s[j], sl2, neg_m));
-                float p1 = ex2(fmaf(s[j + 1], sl2, neg_m));
-                float p2 = ex2(fmaf(s[j + 2], sl2, neg_m));
-                float p3 = ex2(fmaf(s[j + 3], sl2, neg_m));
-                rs4[0] += p0;
-                rs4[1] += p1;
-                rs4[2] += p2;
-                rs4[3] += p3;
-                p[j >> 1] = pack_bf16(p0, p1);
-                p[(j >> 1) + 1] = pack_bf16(p2, p3);
+            for (int j = 0; j < BN; j += 4) {
+                const float2 x01 = __ffma2_rn(make_float2(s[j], s[j + 1]), sl2_2, neg_m);
+                const float2 x23 = __ffma2_rn(make_float2(s[j + 2], s[j + 3]), sl2_2, neg_m);
+                const float2 e01 = make_float2(ex2(x01.x), ex2(x01.y));  // special-function unit
+                const float2 e23 = exp2_fma(x23);                         // FMA pipe
+                rs_a = __fadd2_rn(rs_a, e01);
+                rs_b = __fadd2_rn(rs_b, e23);
+                p[j >> 1] = pack_bf16_int(e01.x, e01.y);
+                p[(j >> 1) + 1] = pack_bf16_int(e23.x, e23.y);
             }
-            l_run = l_run * alpha + ((rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
+            l_run = l_run * alpha + ((rs_a.x + rs_a.y) + (rs_b.x + rs_b.y));
             // O is rescaled only when some row of this warp moved its reference maximum, and only
             // then must the previous P V be complete (P itself lives in its own S buffer)
             const bool rescale = __any_sync(0xffffffffu, alpha != 1.f);
             if (t > 0 && rescale) {
-                alive = wait(&bars.pv_done, (uint32_t)((t - 1) & 1), abort_flag);
+                alive = wait(&bars.pv_done[qt], (uint32_t)((t - 1) & 1), abort_flag);
                 alive = __all_sync(0xffffffffu, alive);
                 if (!alive)
                     break;
                 tc_fence_after();
 #pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2) {
+                for (int c4 = 0; c4 < 4; ++c4) {
                     uint32_t v[32];
-                    tmem_ld32(tmem + lane_addr + COL_O + half * 64 + c2 * 32, v);
+                    tmem_ld32(tbase + COL_O + c4 * 32, v);
                     tmem_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
                         v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
-                    tmem_st32(tmem + lane_addr + COL_O + half * 64 + c2 * 32, v);
+                    tmem_st32(tbase + COL_O + c4 * 32, v);
                 }
                 tmem_wait_st();
             }
-            // P row (bf16 pairs): keys 64*half.. of the tile = packed columns 32*half.. of the S buffer
-            tmem_st32(sa + half * (HN / 2), p);
+            // P row (64 bf16 = 32 packed columns) over the start of its own S buffer
+            tmem_st32(sa, p);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(&bars.p_full);
+            mbar_arrive(&bars.p_full[qt]);
         }
-        if (alive) {
-            // row sums of the two halves meet in shared memory
-            s_rowmax[ntiles & 1][half][row] = l_run;
-            mbar_arrive(&bars.x_full);
-            alive = wait(&bars.x_full, (uint32_t)(ntiles & 1), abort_flag);
+        // A parity wait is only meaningful one phase back.  Waits on pv_done are skipped whenever no
+        // rescale is needed, so catch up one phase at a time: S of the last tile being complete implies
+        // the P V of tile ntiles-3 is, i.e. the barrier is at most two phases behind here.
+        if (alive && ntiles >= 2) {
+            alive = wait(&bars.pv_done[qt], (uint32_t)((ntiles - 2) & 1), abort_flag);
             alive = __all_sync(0xffffffffu, alive);
         }
         if (alive) {
-            alive = wait(&bars.pv_done, (uint32_t)((ntiles - 1) & 1), abort_flag);
+            alive = wait(&bars.pv_done[qt], (uint32_t)((ntiles - 1) & 1), abort_flag);
             alive = __all_sync(0xffffffffu, alive);
         }
         if (alive) {
             tc_fence_after();
-            const float inv = 1.f / (l_run + s_rowmax[ntiles & 1][half ^ 1][row]);
-            const bool ok = row < nrows;
-            const int tok = ok ? (rowlist ? rowlist[row] : row0 + row) : 0;
-            bf16 *orow = Oh + (int64_t)tok * a.sn + half * 64;
+            const float inv = 1.f / l_run;
+            const int gr = qt * BM + row;
+            const bool ok = gr < nrows;
+            const int tok = ok ? (rowlist ? rowlist[gr] : row0 + gr) : 0;
+            bf16 *orow = Oh + (int64_t)tok * a.sn;
 #pragma unroll
-            for (int c2 = 0; c2 < 2; ++c2) {
+            for (int c4 = 0; c4 < 4; ++c4) {
                 uint32_t v[32];
-                tmem_ld32(tmem + lane_addr + COL_O + half * 64 + c2 * 32, v);
+                tmem_ld32(tbase + COL_O + c4 * 32, v);
                 tmem_wait_ld();
                 if (ok) {
 #pragma unroll
@@ -407,7 +440,7 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
                         o.y = pack_bf16(__uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv);
                         o.z = pack_bf16(__uint_as_float(v[j + 4]) * inv, __uint_as_float(v[j + 5]) * inv);
                         o.w = pack_bf16(__uint_as_float(v[j + 6]) * inv, __uint_as_float(v[j + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(orow + c2 * 32 + j) = o;
+                        *reinterpret_cast<uint4 *>(orow + c4 * 32 + j) = o;
                     }
                 }
             }

@@ -102,7 +102,7 @@ void launch_select(const SelectArgs &a, cudaStream_t st);
 void launch_group(const GroupArgs &a, cudaStream_t st);
 void launch_tiles_from_offsets(const GroupArgs &a, cudaStream_t st);
 void launch_attn(const AttnArgs &a, cudaStream_t st);
-constexpr int kAttnTileRows = 128;
+constexpr int kAttnTileRows = 256;
 
 void count_launch(int n = 1);
 
