@@ -12,8 +12,7 @@
 //   * 2 x 4 softmax warps, one thread per query row (= TMEM lane): read S, keep the running row
 //     maximum and row sum in registers, rescale O in tensor memory when the maximum has grown by
 //     more than 2^8, write P (bf16) over their S buffer in tensor memory, from where it is the A
-//     operand of the second MMA.  Half of the exponentials run on the FMA pipe (range reduction +
-//     polynomial) because the special-function unit alone is slower than the tensor core here.
+//     operand of the second MMA.
 // Roles synchronise through mbarriers only; every wait is bounded and a time-out ends the block
 // with an error status instead of hanging.
 #include "scope_internal.cuh"
@@ -77,33 +76,6 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
-// 2^x for two values on the FMA pipe: x = n + f with n integer and |f| <= 1/2 (magic-number
-// rounding), 2^f by a degree-4 polynomial (relative error 4e-5, far below bf16 resolution), n added
-// into the exponent field.  x is clamped at -126 (the result is then ~1e-38, i.e. no weight).
-__device__ __forceinline__ float2 exp2_fma(float2 x)
-{
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
-    const float2 magic = make_float2(12582912.f, 12582912.f);
-    const float2 r = __fadd2_rn(x, magic);
-    const float2 n = __fadd2_rn(r, make_float2(-12582912.f, -12582912.f));
-    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
-    float2 p = __ffma2_rn(f, make_float2(9.6181291e-3f, 9.6181291e-3f), make_float2(5.5504109e-2f, 5.5504109e-2f));
-    p = __ffma2_rn(p, f, make_float2(2.4022651e-1f, 2.4022651e-1f));
-    p = __ffma2_rn(p, f, make_float2(6.9314718e-1f, 6.9314718e-1f));
-    p = __ffma2_rn(p, f, make_float2(1.f, 1.f));
-    float2 y;
-    y.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(r.x) << 23));
-    y.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23));
-    return y;
-}
-
-// two non-negative floats -> packed bf16 pair, round half up (differs from round-to-nearest-even
-// only on exact ties), on the integer pipe
-__device__ __forceinline__ uint32_t pack_bf16_int(float lo, float hi)
-{
-    return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
-}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -374,12 +346,12 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
             for (int j = 0; j < BN; j += 4) {
                 const float2 x01 = __ffma2_rn(make_float2(s[j], s[j + 1]), sl2_2, neg_m);
                 const float2 x23 = __ffma2_rn(make_float2(s[j + 2], s[j + 3]), sl2_2, neg_m);
-                const float2 e01 = make_float2(ex2(x01.x), ex2(x01.y));  // special-function unit
-                const float2 e23 = exp2_fma(x23);                         // FMA pipe
+                const float2 e01 = make_float2(ex2(x01.x), ex2(x01.y));
+                const float2 e23 = make_float2(ex2(x23.x), ex2(x23.y));
                 rs_a = __fadd2_rn(rs_a, e01);
                 rs_b = __fadd2_rn(rs_b, e23);
-                p[j >> 1] = pack_bf16_int(e01.x, e01.y);
-                p[(j >> 1) + 1] = pack_bf16_int(e23.x, e23.y);
+                p[j >> 1] = pack_bf16(e01.x, e01.y);
+                p[(j >> 1) + 1] = pack_bf16(e23.x, e23.y);
             }
             l_run = l_run * alpha + ((rs_a.x + rs_a.y) + (rs_b.x + rs_b.y));
             // O is rescaled only when some row of this warp moved its reference maximum, and only

@@ -57,7 +57,8 @@ __global__ void pack_codes_kernel(uint32_t *codes, const int32_t *src, int64_t n
             bad = true;
             v = 0;
         }
-        codes[i] = (codes[i] & ~(kCodeMask << sh)) | ((uint32_t)v << sh);
+        // the two bits above the three fields stay clear whatever the word held before
+        codes[i] = (codes[i] & ~(kCodeMask << sh) & 0x3fffffffu) | ((uint32_t)v << sh);
     }
     if (__syncthreads_or(bad) && threadIdx.x == 0)
         atomicCAS(status + ST_CODE, 0, (int)SCOPE_ERR_BAD_PLAN);

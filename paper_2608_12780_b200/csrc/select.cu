@@ -45,7 +45,7 @@ __device__ __forceinline__ float proxy_raw(const RowTables &t, uint32_t code)
 {
     // Eq. 6 before the 1/sqrt(d) factor, in this order
     float a = t.T[code & kCodeMask] + t.H[(code >> kCodeBits) & kCodeMask];
-    return a + t.W[code >> (2 * kCodeBits)];
+    return a + t.W[(code >> (2 * kCodeBits)) & kCodeMask];
 }
 
 __device__ __forceinline__ void load_tables(const SelectArgs &a, int bh, int c0, float *lut, RowTables *rt)

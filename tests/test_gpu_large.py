@@ -1,0 +1,85 @@
+"""Full-size configurations (the launch configurations the benchmark times), checked on sampled
+heads and rows the CPU oracle can compute one by one.
+
+Per sampled head: the end-to-end plan of the CUDA path against the oracle's (labels, counts,
+per-head k, key sets), the selection stage fed the oracle's codes / tables / cluster sizes
+(selected-mask Jaccard >= 0.999 per cluster, the bar for large shapes), and the attention output of
+sampled query rows given the CUDA path's own key sets (max-abs 2e-2, relative L2 1e-2).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import scope_oracle as orc
+from paper_2608_12780_b200 import binding as sb
+from paper_2608_12780_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _jaccard(a, b):
+    inter = np.intersect1d(a, b, assume_unique=True).shape[0]
+    return inter / (a.shape[0] + b.shape[0] - inter)
+
+
+@pytest.mark.parametrize("name,heads", [("W480", (0, 17)), ("W720", (5,)), ("HY720", (3, 23))])
+def test_full_size_layer_on_sampled_heads(name, heads):
+    cfg = inputs.CONFIGS[name]
+    Q, K, V = inputs.make_qkv(cfg, seed=0, threads=16)
+    dQ, dK, dV = (sb.bits_to_torch(x, device="cuda") for x in (Q, K, V))
+    plan = sb.Plan(sb.make_params(cfg))
+    O = sb.scope_forward(dQ, dK, dV, plan)
+    plan.check()
+    O = O[0].float().cpu().numpy()
+    g = plan.export("Q_ASSIGN")
+    n_c = plan.export("CLUSTER_SIZES")
+    t_c, r_c, k_head = plan.export("TOPP_COUNT"), plan.export("FINAL_COUNT"), plan.export("K_HEAD")
+    off, idx = plan.export("KEY_OFFSETS"), plan.export("KEY_INDICES")
+    codes = [plan.export(f"K_CODES_{m}") for m in "THW"]
+    perm, qoff = plan.export("Q_PERM"), plan.export("Q_OFFSETS")
+    Cq, N = cfg.Cq, cfg.N
+
+    # structure that holds at any size, all heads
+    assert np.array_equal(n_c.sum(1), np.full(cfg.H, N))
+    assert np.all(r_c >= k_head[:, None]) and np.all(k_head >= cfg.k_fix) and np.all(r_c <= N)
+    assert np.array_equal(np.diff(off), r_c.reshape(-1))
+    for h in heads:
+        assert np.array_equal(np.sort(perm[h]), np.arange(N))
+        assert np.array_equal(g[h][perm[h]], np.repeat(np.arange(Cq), n_c[h]))
+
+    ref = orc.plan_layer(Q[:, list(heads)], K[:, list(heads)], cfg, threads=len(heads))
+    sub = sb.Plan(sb.make_params(cfg, H=len(heads)))
+    st = lambda f: np.stack([f(p) for p in ref])
+    for m, mn in enumerate("THW"):
+        sub.import_(f"K_CODES_{mn}", st(lambda p: p.z[m]))
+        sub.import_(f"LUT_{mn}", st(lambda p: p.P[m]))
+    sub.import_("CLUSTER_SIZES", st(lambda p: p.n_c))
+    sb.scope_plan_stages(None, None, sub, sb.STAGE_SELECT)
+    sub.check()
+    soff, sidx = sub.export("KEY_OFFSETS"), sub.export("KEY_INDICES")
+    assert np.array_equal(sub.export("K_HEAD"), np.array([p.k_head for p in ref]))
+    assert np.array_equal(sub.export("TOPP_COUNT"), st(lambda p: p.t_c))
+
+    rng = np.random.default_rng(1)
+    for i, h in enumerate(heads):
+        p = ref[i]
+        # selection given the oracle's upstream arrays: the large-shape bar, per cluster
+        for c in range(Cq):
+            S = sidx[soff[i * Cq + c]: soff[i * Cq + c + 1]]
+            assert _jaccard(S, p.S[c]) >= 0.999, (name, h, c)
+        # the whole plan, end to end (decisions far from a coin toss are reproduced exactly)
+        assert p.kmeans_gap > 1e-12 and p.topp_margin > 1e-13
+        assert np.array_equal(g[h], p.g), f"{name} head {h}: {(g[h] != p.g).sum()} query labels differ"
+        for m in range(3):
+            assert np.array_equal(codes[m][h], p.z[m]), f"{name} head {h}: key codes {m} differ"
+        assert np.array_equal(t_c[h], p.t_c) and k_head[h] == p.k_head and np.array_equal(r_c[h], p.r_c)
+        for c in rng.choice(Cq, 12, replace=False):
+            S = idx[off[h * Cq + c]: off[h * Cq + c + 1]]
+            assert np.array_equal(S, p.S[c]), (name, h, c)
+        # attention rows given the identical plan
+        rows = rng.choice(N, 48, replace=False)
+        Sg = [idx[off[h * Cq + c]: off[h * Cq + c + 1]] for c in range(Cq)]
+        Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], g[h], Sg, cfg.scale, rows)
+        err = np.abs(O[h][rows] - Oref).max()
+        rel = np.linalg.norm(O[h][rows] - Oref) / np.linalg.norm(Oref)
+        assert err <= 2e-2 and rel <= 1e-2, (name, h, err, rel)

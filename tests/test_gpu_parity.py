@@ -178,6 +178,9 @@ def test_stages_teacher_forced(name, seed):
     Q, K, V, dQ, dK, dV = _layer(cfg, seed)
     ref = _oracle_plans(Q, K, cfg)
     plan = sb.Plan(sb.make_params(cfg))
+    # imports must not depend on what the workspace held before (e.g. the spare bits of the packed codes)
+    plan.workspace.fill_(255)
+    plan.reset_status()
     _import_upstream(plan, ref, "lut")
     sb.scope_plan_stages(None, None, plan, sb.STAGE_LUT)
     _compare_plan(plan, ref, cfg, what=("lut",))
@@ -321,3 +324,32 @@ def test_large_codebooks_use_general_kernel():
     sb.scope_plan(dQ, dK, plan)
     plan.check()
     _compare_plan(plan, ref, cfg)
+
+
+@pytest.mark.parametrize("Cq,top_p,k_fix", [(1, 0.9, 700), (2, 0.5, 300), (3, 0.97, 64)])
+def test_large_clusters_two_query_tiles_per_block(Cq, top_p, k_fix):
+    """Clusters of several hundred queries: blocks of 256 queries with both query tiles in use, many key
+    tiles, ragged last block and ragged last key tile."""
+    cfg = inputs.CONFIGS["small"].replace(H=2, Cq=Cq, top_p=top_p, k_fix=k_fix)
+    Q, K, V, dQ, dK, dV = _layer(cfg, 11)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.H * cfg.Cq * cfg.N))
+    O = _to_np(sb.scope_forward(dQ, dK, dV, plan))
+    plan.check()
+    ref = _oracle_plans(Q, K, cfg)
+    _compare_plan(plan, ref, cfg)
+    for h in range(cfg.H):
+        Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], ref[h].g, ref[h].S, cfg.scale, np.arange(cfg.N))
+        err, rel = _attn_errors(O[0, h], Oref)
+        assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (h, err, rel)
+
+
+def test_dense_mode_many_blocks():
+    cfg = inputs.CONFIGS["small"].replace(H=2)
+    Q, K, V, dQ, dK, dV = _layer(cfg, 12)
+    plan = sb.Plan(sb.make_params(cfg))
+    Od = _to_np(sb.scope_dense_attn(dQ, dK, dV, plan))
+    rows = np.arange(0, cfg.N, 5)
+    for h in range(cfg.H):
+        ref = orc.dense_rows(Q[0, h], K[0, h], V[0, h], cfg.scale, rows)
+        err, rel = _attn_errors(Od[0, h][rows], ref)
+        assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (h, err, rel)
