@@ -56,15 +56,34 @@ __host__ __device__ inline bool tc_layout(const KmArgs &a, TcLayout &L)
     return col <= TMEM_COLS_PER_GROUP;
 }
 
+constexpr int MAXC = 256;  // centroids per range this kernel holds
+
 struct GroupShared {
-    int asg[3][TM];
-    uint32_t sorted[3][TM];
-    float x2[3][TM];
+    int asg[3][TM];              // label of every token of the tile, per range
+    int pos[3][TM];              // slot of the token inside its label's run
+    int cnt[3][MAXC];            // members per label in this tile
+    int start[3][MAXC];          // first slot of the label's run
+    uint32_t runs[3][TM];        // non-empty labels: label | start << 10 | count << 18
+    int nruns[3];
+    uint8_t sorted[3][TM];       // tokens of the tile grouped by label
+    float x2[TM];                // squared norm of the token's row
     int flagged[3 * TM];
     int nflagged;
     int dead;
     uint64_t mbar;
 };
+
+__device__ __forceinline__ void load_x_tile(const KmArgs &a, const bf16 *Xh, int tok0, uint32_t xbase, int gt)
+{
+    // 128 rows x 16 chunks of 16 bytes; rows past N are zero
+    for (int e = gt; e < TM * 16; e += 128) {
+        int row = e >> 4, chunk = e & 15;
+        bool ok = tok0 + row < a.N;
+        const bf16 *src = Xh + (int64_t)(ok ? tok0 + row : 0) * a.sn + chunk * 8;
+        cp_async16_zfill(xbase + (chunk >> 3) * HALF_BYTES + sw128(row, chunk & 7), src, ok ? 16 : 0);
+    }
+    cp_async_commit();
+}
 
 __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int tiles_per_block, int32_t *status)
 {
@@ -82,6 +101,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int grp = tid >> 7, gt = tid & 127;       // pipeline, thread within it
+    const int gw = warp & 3;                        // warp within the pipeline = TMEM lane quarter
     const int bh = blockIdx.y;
     const int b = bh / a.H, h = bh % a.H;
     const bf16 *Xh = a.X + (int64_t)b * a.sb + (int64_t)h * a.sh;
@@ -112,70 +132,69 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             s_un[L.un_off[s] + e] = e < a.sp[s].C ? a.sp[s].unorm[(size_t)bh * a.sp[s].C + e] : INFINITY;
     }
     cp_async_commit();
+    const uint32_t tmem = s_tmem_base + grp * TMEM_COLS_PER_GROUP;  // read after the barrier below
+    const uint32_t xbase = smem_u32(s_x) + grp * XTILE_BYTES;
+    const int ntiles = (a.N + TM - 1) / TM;
+    const int first = blockIdx.x * tiles_per_block + grp;
+    const int last = min(ntiles, (int)(blockIdx.x + 1) * tiles_per_block);  // exclusive
     cp_async_wait<0>();
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = s_tmem_base + grp * TMEM_COLS_PER_GROUP;
-    const uint32_t xbase = smem_u32(s_x) + grp * XTILE_BYTES;
-    const int ntiles = (a.N + TM - 1) / TM;
+    const uint32_t tmem_g = *reinterpret_cast<volatile uint32_t *>(&s_tmem_base) + grp * TMEM_COLS_PER_GROUP;
+    (void)tmem;
     uint32_t phase = 0;
     bool dead = false;
+    // descriptor words: high word fixed, low word = start address
+    const uint64_t d0 = smem_desc_sw128(0);
+    const uint32_t d_hi = (uint32_t)(d0 >> 32), d_lo = (uint32_t)d0;
 
-    for (int ti = grp; ti < tiles_per_block; ti += GROUPS) {
-        const int tile = blockIdx.x * tiles_per_block + ti;
-        if (tile >= ntiles || dead)
-            break;
+    for (int tile = first; tile < last && !dead; tile += GROUPS) {
         const int tok0 = tile * TM;
-        if (gt == 0)
-            G.nflagged = 0;
-        // X tile: 128 rows x 16 chunks; rows past N are zero
-        for (int e = gt; e < TM * 16; e += 128) {
-            int row = e >> 4, chunk = e & 15;
-            bool ok = tok0 + row < a.N;
-            const bf16 *src = Xh + (int64_t)(ok ? tok0 + row : 0) * a.sn + chunk * 8;
-            cp_async16_zfill(xbase + (chunk >> 3) * HALF_BYTES + sw128(row, chunk & 7), src, ok ? 16 : 0);
-        }
-        cp_async_commit();
+        const bool valid = tok0 + gt < a.N;
+        load_x_tile(a, Xh, tok0, xbase, gt);
         cp_async_wait<0>();
         fence_proxy_async();
         tc_fence_before();
         bar_sync(1 + grp, 128);
+        // ---- distances on the tensor core: one thread issues, the others take the row norms meanwhile
         if (gt == 0) {
             tc_fence_after();
+            G.nflagged = 0;
             for (int s = 0; s < a.nspaces; ++s) {
                 const int cp = L.cpad[s];
                 const uint32_t idesc = idesc_bf16(TM, cp, false, false);
                 const int k_lo = a.sp[s].ch0 >> 4, k_hi = (a.sp[s].ch0 + a.sp[s].D + 15) >> 4;
-                bool first = true;
+                const uint32_t cb = smem_u32(s_cent) + L.cent_off[s];
+                bool acc = false;
                 for (int p = 0; p < 3; ++p)
                     for (int ks = k_lo; ks < k_hi; ++ks) {
-                        uint64_t da = smem_desc_sw128(xbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32);
-                        uint64_t db = smem_desc_sw128(smem_u32(s_cent) + L.cent_off[s] + (p * 2 + (ks >> 2)) * cp * 128 + (ks & 3) * 32);
-                        mma_ss(tmem + L.col[s], da, db, idesc, !first);
-                        first = false;
+                        const uint32_t ao = (xbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4;
+                        const uint32_t bo = (cb + (p * 2 + (ks >> 2)) * cp * 128 + (ks & 3) * 32) >> 4;
+                        mma_ss2(tmem_g + L.col[s], d_lo + ao, d_hi, d_lo + bo, d_hi, idesc, acc);
+                        acc = true;
                     }
             }
             mma_commit(&G.mbar);
         }
-        // squared norm of the token's slice per space while the MMAs run
+        for (int e = gt; e < a.nspaces * MAXC; e += 128)
+            (&G.cnt[0][0])[e] = 0;
         {
-            float x2[3] = {0.f, 0.f, 0.f};
+            // squared norm of the whole row (an upper bound of every range's slice, used in the tolerance)
+            float x2a = 0.f, x2b = 0.f;
 #pragma unroll
             for (int chunk = 0; chunk < 16; ++chunk) {
                 uint4 raw = *reinterpret_cast<const uint4 *>(s_x + grp * XTILE_BYTES + (chunk >> 3) * HALF_BYTES + sw128(gt, chunk & 7));
-                const bf16 *e = reinterpret_cast<const bf16 *>(&raw);
+                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    int ch = chunk * 8 + q;
-                    float v = __bfloat162float(e[q]);
-                    int s = (a.nspaces == 1 || ch < a.sp[1].ch0) ? 0 : (ch < a.sp[2].ch0 ? 1 : 2);
-                    x2[s] = fmaf(v, v, x2[s]);
+                for (int q = 0; q < 4; ++q) {
+                    float lo = __uint_as_float(w[q] << 16), hi = __uint_as_float(w[q] & 0xffff0000u);
+                    x2a = fmaf(lo, lo, x2a);
+                    x2b = fmaf(hi, hi, x2b);
                 }
             }
-            for (int s = 0; s < a.nspaces; ++s)
-                G.x2[s][gt] = x2[s];
+            G.x2[gt] = x2a + x2b;
         }
         // a wait that runs out is recorded and ends this pipeline after the next barrier
         const bool ok = __all_sync(0xffffffffu, mbar_wait(&G.mbar, phase));
@@ -186,24 +205,44 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         phase ^= 1;
         tc_fence_after();
         if (ok) {
+            const float x2 = G.x2[gt];
             for (int s = 0; s < a.nspaces; ++s) {
-                const int C = a.sp[s].C;
+                const int C = a.sp[s].C, cp = L.cpad[s];
                 const float *un = s_un + L.un_off[s];
+                const uint32_t ta = tmem_g + ((uint32_t)(gw * 32) << 16) + L.col[s];
                 float best = INFINITY, second = INFINITY;
                 int arg = 0;
-                for (int c0 = 0; c0 < L.cpad[s]; c0 += 16) {
-                    uint32_t r[16];
-                    tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + L.col[s] + c0, r);
-                    tmem_wait_ld();
+                for (int c0 = 0; c0 < cp; c0 += 32) {
+                    uint32_t r[32];
+                    if (cp - c0 >= 32) {
+                        tmem_ld32(ta + c0, r);
+                    } else {  // a last group of 16 columns
+                        uint32_t r16[16];
+                        tmem_ld16(ta + c0, r16);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        float dist = fmaf(-2.f, __uint_as_float(r[j]), un[c0 + j]);  // padding columns carry +inf norms
-                        if (dist < best) {
-                            second = best;
-                            best = dist;
-                            arg = c0 + j;
-                        } else if (dist < second) {
-                            second = dist;
+                        for (int j = 0; j < 16; ++j) {
+                            r[j] = r16[j];
+                            r[16 + j] = 0u;
+                        }
+                    }
+                    tmem_wait_ld();
+                    const int nc = min(32, cp - c0);
+#pragma unroll
+                    for (int j4 = 0; j4 < 32; j4 += 4) {
+                        if (j4 < nc) {
+                            const float4 u4 = *reinterpret_cast<const float4 *>(un + c0 + j4);  // padding columns carry +inf
+                            const float uu[4] = {u4.x, u4.y, u4.z, u4.w};
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float dist = fmaf(-2.f, __uint_as_float(r[j4 + q]), uu[q]);
+                                if (dist < best) {
+                                    second = best;
+                                    best = dist;
+                                    arg = c0 + j4 + q;
+                                } else if (dist < second) {
+                                    second = dist;
+                                }
+                            }
                         }
                     }
                 }
@@ -213,8 +252,8 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                 // of the 3 * (channels / 16) accumulating MMAs may lose up to two fp32 ulps of the running
                 // magnitude (truncating adds), |x.u| <= (|u|^2 + |x|^2) / 2; doubled for margin
                 const float kappa = 8.f * (float)(3 * ((cend - cbeg) >> 4) + 2) * 1.1920929e-7f;
-                const float tol = kappa * (__ldg(a.sp[s].u2max + bh) + G.x2[s][gt]);
-                if (tok0 + gt < a.N && C > 1 && second - best <= tol) {
+                const float tol = kappa * (__ldg(a.sp[s].u2max + bh) + x2);
+                if (valid && C > 1 && second - best <= tol) {
                     int slot = atomicAdd(&G.nflagged, 1);
                     G.flagged[slot] = (s << 16) | gt;
                 }
@@ -223,28 +262,40 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         tc_fence_before();
         bar_sync(1 + grp, 128);
         dead = *reinterpret_cast<volatile int *>(&G.dead) != 0;
+        if (dead)
+            break;
 
-        // fp64 re-evaluation of the close calls: one warp per token, centroids spread over lanes
+        // ---- fp64 re-evaluation of the close calls: one warp per token, four centroids per lane at a time.
+        // Every centroid's distance is summed in the same fixed order, so equal centroids tie exactly and
+        // the lowest index wins, as in a plain sequential evaluation.
         {
-            const int nf = dead ? 0 : G.nflagged;
-            for (int f = (warp & 3); f < nf; f += 4) {
+            const int nf = G.nflagged;
+            for (int f = gw; f < nf; f += 4) {
                 const int s = G.flagged[f] >> 16, lt = G.flagged[f] & 0xffff;
                 const KmSpace &sp = a.sp[s];
                 const float *cent = sp.cent + (size_t)bh * sp.C * sp.D;
                 const bf16 *x = Xh + (int64_t)(tok0 + lt) * a.sn + sp.ch0;
                 double bd = INFINITY;
                 int ba = 0x7fffffff;
-                for (int c = lane; c < sp.C; c += 32) {
-                    const float *u = cent + (size_t)c * sp.D;
-                    double dist = 0.0;
+                for (int c = lane; c < sp.C; c += 128) {
+                    const int c1 = min(c + 32, sp.C - 1), c2 = min(c + 64, sp.C - 1), c3 = min(c + 96, sp.C - 1);
+                    const float *u0 = cent + (size_t)c * sp.D, *u1 = cent + (size_t)c1 * sp.D;
+                    const float *u2 = cent + (size_t)c2 * sp.D, *u3 = cent + (size_t)c3 * sp.D;
+                    double d0 = 0.0, d1 = 0.0, d2 = 0.0, d3 = 0.0;
                     for (int ch = 0; ch < sp.D; ++ch) {
-                        double diff = __dsub_rn((double)__bfloat162float(x[ch]), (double)u[ch]);
-                        dist = __dadd_rn(dist, __dmul_rn(diff, diff));
+                        const double xv = (double)__bfloat162float(x[ch]);
+                        double e0 = __dsub_rn(xv, (double)u0[ch]), e1 = __dsub_rn(xv, (double)u1[ch]);
+                        double e2 = __dsub_rn(xv, (double)u2[ch]), e3 = __dsub_rn(xv, (double)u3[ch]);
+                        d0 = __dadd_rn(d0, __dmul_rn(e0, e0));
+                        d1 = __dadd_rn(d1, __dmul_rn(e1, e1));
+                        d2 = __dadd_rn(d2, __dmul_rn(e2, e2));
+                        d3 = __dadd_rn(d3, __dmul_rn(e3, e3));
                     }
-                    if (dist < bd) {
-                        bd = dist;
-                        ba = c;
-                    }
+                    // ascending index order keeps the lowest index on ties
+                    if (d0 < bd) { bd = d0; ba = c; }
+                    if (c + 32 < sp.C && d1 < bd) { bd = d1; ba = c + 32; }
+                    if (c + 64 < sp.C && d2 < bd) { bd = d2; ba = c + 64; }
+                    if (c + 96 < sp.C && d3 < bd) { bd = d3; ba = c + 96; }
                 }
 #pragma unroll
                 for (int m = 16; m >= 1; m >>= 1) {
@@ -260,28 +311,54 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             }
         }
         bar_sync(1 + grp, 128);
-        if (dead)
-            break;
 
-        // labels out
-        if (tok0 + gt < a.N) {
-            if (a.nspaces == 1)
-                a.assign[(size_t)bh * a.N + tok0 + gt] = G.asg[0][gt];
-            else
-                a.codes[(size_t)bh * a.N + tok0 + gt] = (uint32_t)G.asg[0][gt] | ((uint32_t)G.asg[1][gt] << kCodeBits) |
-                                                        ((uint32_t)G.asg[2][gt] << (2 * kCodeBits));
-        }
-        // order the tile's tokens by label (rank by counting), then add each run of equal labels once
-        for (int s = 0; s < a.nspaces; ++s) {
-            uint32_t key = (tok0 + gt < a.N ? (uint32_t)G.asg[s][gt] : (uint32_t)kMaxClusters) << 8 | (uint32_t)gt;
-            int rank = 0;
-            for (int o = 0; o < TM; ++o) {
-                uint32_t ok = (tok0 + o < a.N ? (uint32_t)G.asg[s][o] : (uint32_t)kMaxClusters) << 8 | (uint32_t)o;
-                rank += ok < key;
+        // ---- labels out, and the tile's tokens grouped by label (counting sort in shared memory)
+        int lab[3] = {0, 0, 0};
+        if (valid) {
+            for (int s = 0; s < a.nspaces; ++s) {
+                lab[s] = G.asg[s][gt];
+                G.pos[s][gt] = atomicAdd(&G.cnt[s][lab[s]], 1);
             }
-            G.sorted[s][rank] = key;
+            if (a.nspaces == 1)
+                a.assign[(size_t)bh * a.N + tok0 + gt] = lab[0];
+            else
+                a.codes[(size_t)bh * a.N + tok0 + gt] =
+                    (uint32_t)lab[0] | ((uint32_t)lab[1] << kCodeBits) | ((uint32_t)lab[2] << (2 * kCodeBits));
         }
         bar_sync(1 + grp, 128);
+        if (gw < a.nspaces) {
+            // one warp per range: exclusive scan of the counts, list of the non-empty labels
+            const int s = gw, cp = L.cpad[s];
+            int base = 0, nr = 0;
+            for (int c0 = 0; c0 < cp; c0 += 32) {
+                const int c = c0 + lane;
+                const int n = c < cp ? G.cnt[s][c] : 0;
+                int inc = n;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    int v = __shfl_up_sync(0xffffffffu, inc, o);
+                    if (lane >= o)
+                        inc += v;
+                }
+                const int st = base + inc - n;
+                if (c < cp)
+                    G.start[s][c] = st;
+                const uint32_t m = __ballot_sync(0xffffffffu, n > 0);
+                if (n > 0)
+                    G.runs[s][nr + __popc(m & ((1u << lane) - 1u))] = (uint32_t)c | ((uint32_t)st << 10) | ((uint32_t)n << 18);
+                nr += __popc(m);
+                base += __shfl_sync(0xffffffffu, inc, 31);
+            }
+            if (lane == 0)
+                G.nruns[s] = nr;
+        }
+        bar_sync(1 + grp, 128);
+        if (valid)
+            for (int s = 0; s < a.nspaces; ++s)
+                G.sorted[s][G.start[s][lab[s]] + G.pos[s][gt]] = (uint8_t)gt;
+        bar_sync(1 + grp, 128);
+
+        // ---- member sums: one thread per channel, one fp64 atomic per (label present in the tile, channel)
         {
             const int ch = gt;
             int s = 0;
@@ -293,35 +370,34 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             int32_t *counts = sp.counts + (size_t)bh * sp.C;
             const unsigned char *xcol = s_x + grp * XTILE_BYTES + (ch >> 6) * HALF_BYTES + (ch & 7) * 2;
             const int chunk = (ch & 63) >> 3;
-            int cur = -1, run = 0;
-            double acc = 0.0;
-            for (int l = 0; l < TM; ++l) {
-                uint32_t key = G.sorted[s][l];
-                int cl = (int)(key >> 8), lt = (int)(key & 255u);
-                if (cl >= kMaxClusters)
-                    break;
-                if (cl != cur) {
-                    if (cur >= 0) {
-                        atomicAdd(sums + (size_t)cur * sp.D + rel, acc);
-                        if (rel == 0)
-                            atomicAdd(counts + cur, run);
-                    }
-                    cur = cl;
-                    acc = 0.0;
-                    run = 0;
+            const int nr = G.nruns[s];
+            for (int r = 0; r < nr; ++r) {
+                const uint32_t run = G.runs[s][r];
+                const int cl = run & 1023, st = (run >> 10) & 255, n = run >> 18;
+                const uint8_t *tok = &G.sorted[s][st];
+                double acc0 = 0.0, acc1 = 0.0;
+                int l = 0;
+                for (; l + 8 <= n; l += 8) {
+                    float v[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        v[q] = __bfloat162float(*reinterpret_cast<const bf16 *>(xcol + sw128(tok[l + q], chunk)));
+                    // bf16 values of any magnitudes do not add exactly in fp32; in fp64 they do
+                    acc0 += (((double)v[0] + (double)v[1]) + ((double)v[2] + (double)v[3]));
+                    acc1 += (((double)v[4] + (double)v[5]) + ((double)v[6] + (double)v[7]));
                 }
-                acc += (double)__bfloat162float(*reinterpret_cast<const bf16 *>(xcol + sw128(lt, chunk)));
-                ++run;
-            }
-            if (cur >= 0) {
-                atomicAdd(sums + (size_t)cur * sp.D + rel, acc);
+                for (; l < n; ++l)
+                    acc0 += (double)__bfloat162float(*reinterpret_cast<const bf16 *>(xcol + sw128(tok[l], chunk)));
+                atomicAdd(sums + (size_t)cl * sp.D + rel, acc0 + acc1);
                 if (rel == 0)
-                    atomicAdd(counts + cur, run);
+                    atomicAdd(counts + cl, n);
             }
         }
+        tc_fence_before();
         bar_sync(1 + grp, 128);  // the X tile and the label arrays are reused by the next tile
     }
 
+    cp_async_wait<0>();
     tc_fence_before();
     __syncthreads();
     if (warp == 0)
