@@ -31,6 +31,11 @@ from paper_2608_12780_b200 import inputs  # noqa: E402
 
 METRIC = "SCOPE attn-layer ms at 118.8K tokens; sparse-attn TFLOP/s; select GB/s"
 
+# DRAM traffic of one sparse_attn_kernel launch, from the ncu capture summarised in
+# profiles/sparse_attn_kernel_w480_8heads.txt (dram__bytes_read.sum + dram__bytes_write.sum on a case of
+# 8 x 32760 tokens); Q, K, V and O are each touched once, so it is scaled by the token count of the launch.
+ATTN_TRAFFIC_CAPTURE = {"bytes": 233.08e6, "tokens": 8 * 32760}
+
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -45,15 +50,16 @@ def measured_peaks():
 # --------------------------------------------------------------------------------------- CPU oracle arm
 
 
-def oracle_sample(cfg, seed=0):
+def oracle_sample(cfg, seed=0, scale=1.0):
     """Time the oracle, as it stands, single-threaded, on a bounded sample of one layer and
     extrapolate to ms per layer: one Lloyd iteration of one head (queries and the three key
-    ranges), the tables, the selection of 8 query clusters and the attention of 128 query rows."""
+    ranges) for three iterations, the tables, the selection of 32 query clusters and the attention of 256
+    query rows."""
     from oracle import scope_oracle as orc
 
     Q, K, V = inputs.make_head(cfg, seed, 0, 0)
     N, d = cfg.N, cfg.d
-    it_s = min(2, cfg.iters)
+    it_s = max(1, min(int(round(3 * scale)), cfg.iters))
     t0 = time.perf_counter()
     kq = orc.kmeans(Q, 0, d, cfg.Cq, it_s)
     ranges = ((0, cfg.split[0], cfg.Ct), (cfg.split[0], cfg.split[1], cfg.Ch), (cfg.split[0] + cfg.split[1], cfg.split[2], cfg.Cw))
@@ -63,7 +69,7 @@ def oracle_sample(cfg, seed=0):
     P = tuple(orc.lut(kq.U, ch0, km.U)[0] for (ch0, _, _), km in zip(ranges, ks))
     t_lut = time.perf_counter() - t0
     z = tuple(km.assign for km in ks)
-    rows_sel = min(16, cfg.Cq)
+    rows_sel = max(2, min(int(32 * scale), cfg.Cq))
     t0 = time.perf_counter()
     orders, b = [], []
     for c in range(rows_sel):
@@ -77,7 +83,7 @@ def oracle_sample(cfg, seed=0):
     r = [min(N, max(bc, k_est)) for bc in b]
     S = [orc.key_set(orders[c], r[c]) for c in range(rows_sel)]
     t_sel = time.perf_counter() - t0
-    rows_att = min(128, N)
+    rows_att = max(16, min(int(256 * scale), N))
     g = (np.arange(N) % rows_sel).astype(np.int32)
     t0 = time.perf_counter()
     orc.attention_rows(Q, K, V, g, S, cfg.scale, np.arange(rows_att))
@@ -99,8 +105,10 @@ def run_reference(args, cfg):
     for _ in range(args.warmup):
         pass  # the oracle has no warm-up state worth paying for
     sample = ""
-    for _ in range(max(1, args.steps)):
-        ms, sample = oracle_sample(cfg)
+    steps = max(1, args.steps)
+    scale = min(1.0, 7.0 / steps)  # ~20 s of oracle work per step at full scale: keep the whole run to minutes
+    for _ in range(steps):
+        ms, sample = oracle_sample(cfg, scale=scale)
         vals.append(ms)
     ms = float(np.median(vals))
     line = {
@@ -308,7 +316,9 @@ def run_scope(args, cfg):
                        "k_fix": cfg.k_fix, "layers_per_gpu": 1, "parallelism": f"batch-sharded x{world}, no collective",
                        "l2": "inputs larger than L2 (Q, K, V %d MB each)" % (nbytes >> 20)},
             "roofline": {"bound": "tensor", "kernel": "sparse_attn_kernel", "achieved": achieved, "peak": peak,
-                         "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                         "unit": "TFLOP/s", "frac": achieved / peak,
+                         "traffic": ATTN_TRAFFIC_CAPTURE["bytes"] * cfg.H * cfg.N / ATTN_TRAFFIC_CAPTURE["tokens"],
+                         "traffic_note": "bytes per launch, ncu capture of a smaller case scaled by tokens",
                          "peak_source": f"bf16_tflops_sustained of {peaks['source']}",
                          "flop_per_launch": attn_flop, "ms_per_launch": attn_ms},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
