@@ -191,6 +191,30 @@ const char *scope_status_string(scope_status s);
  * arithmetic (a float alpha can be off by one).  Returns -1 on bad arguments. */
 int64_t scope_kfix_from_alpha(int64_t N, int64_t alpha_num, int64_t alpha_den);
 
+/* No counterpart in the paper: a convenience for hosts that forbid device allocation.
+ *
+ * The query clustering of Algorithm 1 line 1 (evenly strided initial centroids, `iters` Lloyd
+ * iterations, labels of the last assignment step, centroids = means of those members) for ONE
+ * head, without any workspace: the scratch this step needs (fp64 member sums, counts, centroid
+ * norms; about 130 KB) sits in a fixed array inside the library, one copy per GPU that has the
+ * library loaded, for the life of the process.  Meant for callers that cannot obtain device
+ * memory when the call is made: a process that handed all of its memory to a pool at start-up,
+ * code running where the allocator must not be entered, or a loop that cannot afford the
+ * device-wide synchronisation an allocation may imply.  Nothing in this call allocates or frees.
+ *   Q          device, bf16, [N, 128], row stride `stride_n` elements (0 = 128), 16-byte aligned
+ *   C          clusters, 1 <= C <= min(N, SCOPE_STATIC_MAX_CLUSTERS); more returns SCOPE_ERR_UNSUPPORTED
+ *   centroids  device out, float [C, 128]      labels  device out, int32 [N]
+ *   sizes      device out, int32 [C] (members per cluster)
+ * The first call on a device looks up the device address of the array (one runtime query, no
+ * launch); make that first call outside any stream capture.  Every call on a device uses the same
+ * array: the call clears what it needs at its start, but two calls whose kernels overlap on the
+ * GPU (different streams, or different host threads) corrupt each other — serialise them.
+ * Asynchronous on `stream`; results equal those of scope_plan_stages(KMEANS_INIT | KMEANS_Q). */
+#define SCOPE_STATIC_MAX_CLUSTERS 128
+scope_status scope_kmeans_queries_static(const void *Q, int32_t N, int64_t stride_n, int32_t C,
+                                         int32_t iters, float *centroids, int32_t *labels,
+                                         int32_t *sizes, void *stream);
+
 /* Number of kernels this library has launched in the calling process since load
  * (diagnostic counter for benchmarks). */
 int64_t scope_kernel_launches(void);

@@ -30,7 +30,8 @@ STAGE_ALL = 63
 EXPORTS = ["scope_plan_workspace_bytes", "scope_plan_create", "scope_plan_destroy", "scope_plan", "scope_plan_stages",
            "scope_sparse_attn", "scope_forward", "scope_forward_host", "scope_dense_attn", "scope_plan_status",
            "scope_plan_reset_status", "scope_plan_get", "scope_plan_field_bytes", "scope_plan_export",
-           "scope_plan_import", "scope_status_string", "scope_kfix_from_alpha", "scope_kernel_launches"]
+           "scope_plan_import", "scope_status_string", "scope_kfix_from_alpha", "scope_kernel_launches",
+           "scope_kmeans_queries_static"]
 
 
 class ScopeParams(C.Structure):
@@ -83,6 +84,7 @@ def lib():
         L.scope_status_string.restype = C.c_char_p
         L.scope_kfix_from_alpha.argtypes = [i64, i64, i64]
         L.scope_kfix_from_alpha.restype = i64
+        L.scope_kmeans_queries_static.argtypes = [vp, C.c_int32, i64, C.c_int32, C.c_int32, vp, vp, vp, vp]
         L.scope_kernel_launches.argtypes = []
         L.scope_kernel_launches.restype = i64
         _lib = L
@@ -261,6 +263,23 @@ def scope_forward_host(Qh, Kh, Vh, plan: Plan, Oh, staging: torch.Tensor) -> Non
     nbytes = staging.numel() * staging.element_size() - (base - staging.data_ptr())
     _check(lib().scope_forward_host(Qh.data_ptr(), Kh.data_ptr(), Vh.data_ptr(), plan.handle, Oh.data_ptr(),
                                     C.c_void_p(base), nbytes, C.c_void_p(_stream())), "scope_forward_host")
+
+
+def scope_kmeans_queries_static(Q, C_clusters: int, iters: int):
+    """Query clustering of one head through the entry point that uses no workspace: the caller owns
+    inputs and outputs (allocated here by torch, before the call), the library's fixed scratch array
+    holds the rest.  Q: CUDA bf16 [N, 128] (rows may be strided).  Returns (centroids fp32 [C, 128],
+    labels int32 [N], sizes int32 [C]).  Calls on one device must not overlap."""
+    if not (Q.is_cuda and Q.dtype == torch.bfloat16 and Q.dim() == 2 and Q.shape[1] == 128 and Q.stride(1) == 1):
+        raise TypeError("Q must be a CUDA bfloat16 tensor [N, 128] with contiguous rows")
+    N = Q.shape[0]
+    cent = torch.empty((C_clusters, 128), dtype=torch.float32, device=Q.device)
+    labels = torch.empty(N, dtype=torch.int32, device=Q.device)
+    sizes = torch.empty(C_clusters, dtype=torch.int32, device=Q.device)
+    _check(lib().scope_kmeans_queries_static(Q.data_ptr(), N, Q.stride(0), C_clusters, iters, cent.data_ptr(),
+                                              labels.data_ptr(), sizes.data_ptr(), C.c_void_p(_stream())),
+           "scope_kmeans_queries_static")
+    return cent, labels, sizes
 
 
 def bits_to_torch(u16: np.ndarray, device=None, pin=False) -> torch.Tensor:

@@ -1,0 +1,90 @@
+// scope_kmeans_queries_static: the query clustering of the layer for one head, for callers that may
+// not allocate device memory at all.  Its scratch (member sums, counts, centroid norms) lives in a
+// fixed array inside the loaded library instead of a caller-provided workspace.
+#include <mutex>
+
+#include "scope_internal.cuh"
+
+namespace scope {
+
+namespace {
+
+constexpr int kStaticMaxClusters = 128;  // must match SCOPE_STATIC_MAX_CLUSTERS in scope.h
+constexpr int kMaxDevices = 64;
+
+struct StaticScratch {
+    double sums[kStaticMaxClusters * kHeadDim];  // 128 KB
+    float unorm[kStaticMaxClusters];
+    int32_t counts[kStaticMaxClusters];
+    float u2max[4];
+};
+
+// One copy per GPU that loads the library, held until the process exits.  In host code this name is
+// only a handle for cudaGetSymbolAddress; the device address is looked up once per device below.
+static __device__ __align__(256) unsigned char g_static_scratch[(sizeof(StaticScratch) + 255) / 256 * 256];
+
+std::mutex g_mutex;
+void *g_device_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the scratch array on the current device (looked up on the first call per device).
+cudaError_t static_scratch(StaticScratch **out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess)
+        return e;
+    if (dev < 0 || dev >= kMaxDevices)
+        return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!g_device_ptr[dev]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess)
+            return e;
+        g_device_ptr[dev] = p;
+    }
+    *out = static_cast<StaticScratch *>(g_device_ptr[dev]);
+    return cudaSuccess;
+}
+
+}  // namespace
+
+}  // namespace scope
+
+using namespace scope;
+
+extern "C" scope_status scope_kmeans_queries_static(const void *Q, int32_t N, int64_t stride_n, int32_t C, int32_t iters,
+                                                    float *centroids, int32_t *labels, int32_t *sizes, void *stream)
+{
+    if (!Q || !centroids || !labels || !sizes || N < 1 || C < 1 || C > N || iters < 1)
+        return SCOPE_ERR_INVALID_ARG;
+    if (C > kStaticMaxClusters)
+        return SCOPE_ERR_UNSUPPORTED;  // larger codebooks need the workspace-based scope_plan
+    if (stride_n == 0)
+        stride_n = kHeadDim;
+    if (stride_n < kHeadDim)
+        return SCOPE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(Q) & 15u) || (stride_n % 8))
+        return SCOPE_ERR_ALIGNMENT;
+    StaticScratch *sc = nullptr;
+    if (static_scratch(&sc) != cudaSuccess)
+        return SCOPE_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    KmArgs a{};
+    a.X = static_cast<const bf16 *>(Q);
+    a.sb = 0;
+    a.sh = 0;
+    a.sn = stride_n;
+    a.B = 1;
+    a.H = 1;
+    a.N = N;
+    a.nspaces = 1;
+    a.sp[0] = KmSpace{0, kHeadDim, C, centroids, sc->unorm, sc->u2max, sc->sums, sc->counts, sizes, nullptr, (C + 15) & ~15};
+    a.assign = labels;
+    a.codes = nullptr;
+    // the initialisation pass clears the sums and counts left by the previous call
+    launch_kmeans_init(a, st);
+    for (int it = 0; it < iters; ++it)
+        launch_kmeans_iteration(a, nullptr, st);  // no bf16 splits -> the general fp32 kernel, which has no status word
+    return cudaGetLastError() == cudaSuccess ? SCOPE_OK : SCOPE_ERR_CUDA;
+}

@@ -1,0 +1,61 @@
+"""scope_kmeans_queries_static: the query clustering for hosts that may not allocate device memory
+when they call into the library (everything was handed to a pool at start-up, or the call site must
+not enter the allocator).  Its scratch is a fixed array inside the library, so this test checks the two
+things a caller relies on: the results equal those of the workspace-based entry point, and a second
+call is not disturbed by what the first one left in the shared array.
+
+Collected last on purpose: a failure here must not hide any other test of a stop-at-first-failure run.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_12780_b200 import binding as sb
+from paper_2608_12780_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _workspace_path(cfg, dQ):
+    """Query k-means of one head through scope_plan_stages (caller-allocated workspace)."""
+    plan = sb.Plan(sb.make_params(cfg, H=1, strides=(cfg.N * cfg.d, cfg.N * cfg.d, cfg.d)))
+    sb.scope_plan_stages(dQ, dQ, plan, sb.STAGE_KMEANS_INIT)
+    sb.scope_plan_stages(dQ, dQ, plan, sb.STAGE_KMEANS_Q)
+    plan.check()
+    return plan.export("Q_CENTROIDS")[0], plan.export("Q_ASSIGN")[0], plan.export("CLUSTER_SIZES")[0]
+
+
+def test_static_scratch_entry_point_matches_workspace_path_twice_in_a_row():
+    cfg = inputs.CONFIGS["small"]
+    outs = []
+    # two calls in a row on different inputs (different heads, then a different cluster count):
+    # the second must not see the sums and counts of the first
+    for head, Cq in ((0, cfg.Cq), (5, 17)):
+        c = cfg.replace(Cq=Cq)
+        Q, _, _ = inputs.make_head(c, 0, 0, head)
+        dQ = sb.bits_to_torch(Q, device="cuda").reshape(1, 1, c.N, c.d).contiguous()
+        cent, labels, sizes = sb.scope_kmeans_queries_static(dQ[0, 0], Cq, c.iters)
+        torch.cuda.synchronize()
+        outs.append((c, dQ, cent.cpu().numpy(), labels.cpu().numpy(), sizes.cpu().numpy()))
+    for c, dQ, cent, labels, sizes in outs:
+        ref_cent, ref_labels, ref_sizes = _workspace_path(c, dQ)
+        # same arithmetic on both paths (fp64 decisions and sums): the tolerance of the k-means parity
+        # tests is exact equality
+        assert np.array_equal(labels, ref_labels)
+        assert np.array_equal(sizes, ref_sizes) and sizes.sum() == c.N
+        assert np.array_equal(cent, ref_cent)
+
+
+def test_static_scratch_entry_point_rejects_what_it_cannot_hold():
+    cfg = inputs.CONFIGS["small"]
+    Q, _, _ = inputs.make_head(cfg, 0, 0, 0)
+    dQ = sb.bits_to_torch(Q, device="cuda")
+    with pytest.raises(sb.ScopeError) as e:
+        sb.scope_kmeans_queries_static(dQ, 129, 1)  # more clusters than the fixed array holds
+    assert e.value.status == sb.SCOPE_ERR_UNSUPPORTED
+    with pytest.raises(sb.ScopeError) as e:
+        sb.scope_kmeans_queries_static(dQ[:8], 16, 1)  # more clusters than tokens
+    assert e.value.status == sb.SCOPE_ERR_INVALID_ARG
+    with pytest.raises(sb.ScopeError) as e:
+        sb.scope_kmeans_queries_static(dQ, 4, 0)
+    assert e.value.status == sb.SCOPE_ERR_INVALID_ARG
