@@ -33,6 +33,9 @@ struct scope_plan_s {
     double *q_sums, *k_sums[3];
     int32_t *q_counts, *k_counts[3];
     RowState *rows;
+    uint32_t *item_code, *item_weight;
+    int32_t *item_count, *cell_table;
+    int cells;
     int32_t *tile_offsets;
     int32_t *io_scratch;  // [BH, N] staging for packed-code import / export
 };
@@ -126,6 +129,15 @@ void carve(scope_plan_t *pl, unsigned char *base, size_t *total)
     pl->r_c = cv.take<int32_t>(BH * Cq);
     pl->k_head = cv.take<int32_t>(BH);
     pl->rows = cv.take<RowState>(BH * Cq);
+    pl->item_code = cv.take<uint32_t>(BH * N);
+    pl->item_weight = cv.take<uint32_t>(BH * N);
+    pl->item_count = cv.take<int32_t>(BH);
+    {
+        // code spaces up to 2^18 cells are deduplicated through a count table
+        const size_t cells = C[0] * C[1] * C[2];
+        pl->cells = cells <= ((size_t)1 << 18) ? (int)cells : 0;
+        pl->cell_table = cv.take<int32_t>(BH * (size_t)pl->cells);
+    }
     pl->key_offsets = cv.take<int64_t>(BH * Cq + 1);
     pl->q_perm = cv.take<int32_t>(BH * N);
     pl->q_offsets = cv.take<int32_t>(BH * (Cq + 1));
@@ -355,6 +367,8 @@ scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, u
         a.BH = pl->BH; a.N = p.N; a.Cq = p.Cq; a.Ct = p.Ct; a.Ch = p.Ch; a.Cw = p.Cw;
         a.scale = p.scale; a.top_p = p.top_p; a.k_fix = p.k_fix; a.capacity = p.index_capacity;
         a.codes = pl->k_codes;
+        a.item_code = pl->item_code; a.item_weight = pl->item_weight; a.item_count = pl->item_count;
+        a.cell_table = pl->cell_table; a.cells = pl->cells;
         a.lutT = pl->lut[0]; a.lutH = pl->lut[1]; a.lutW = pl->lut[2];
         a.n_c = pl->n_c;
         a.t_c = pl->t_c; a.b_c = pl->b_c; a.r_c = pl->r_c; a.k_head = pl->k_head;

@@ -56,6 +56,11 @@ struct SelectArgs {
     int k_fix;
     int64_t capacity;
     const uint32_t *codes;   // [BH, N]
+    uint32_t *item_code;     // [BH, N] scratch: distinct composite codes of the head ...
+    uint32_t *item_weight;   // [BH, N] scratch: ... and how many keys carry each
+    int32_t *item_count;     // [BH]    scratch: number of items
+    int32_t *cell_table;     // [BH, cells] scratch: keys per cell of the code space (cells > 0 only)
+    int cells;               // Ct*Ch*Cw if the table is used, else 0 (every key is its own item)
     const float *lutT, *lutH, *lutW;  // [BH, Cq, Cm]
     const int32_t *n_c;      // [BH, Cq]
     int32_t *t_c, *b_c, *r_c, *k_head;

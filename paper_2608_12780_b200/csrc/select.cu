@@ -13,6 +13,8 @@
 // The key set is then written by one ordered pass over the keys: everything above the
 // threshold logit, plus the lowest-indexed keys of the threshold group (equal logits are
 // ranked by ascending key index), in ascending key index.
+#include <algorithm>
+
 #include "scope_internal.cuh"
 
 namespace scope {
@@ -161,6 +163,80 @@ __device__ __forceinline__ int descend(const W *w, const uint32_t *cnt, int nb, 
 }
 
 // ---------------------------------------------------------------------------------------------
+// Keys with the same composite code (Eq. 4) have the same proxy logit for every query cluster, so the
+// threshold searches run over the distinct codes of the head, each weighted by its number of keys.
+// With a small code space (C_T C_H C_W cells) the distinct codes come from a count table; otherwise
+// every key is its own item with weight 1.
+__device__ __forceinline__ uint32_t code_cell(uint32_t code, int Ch, int Cw)
+{
+    return ((code & kCodeMask) * Ch + ((code >> kCodeBits) & kCodeMask)) * Cw + ((code >> (2 * kCodeBits)) & kCodeMask);
+}
+
+__global__ void __launch_bounds__(256) dedupe_count_kernel(SelectArgs a)
+{
+    const int bh = blockIdx.y;
+    const uint32_t *codes = a.codes + (size_t)bh * a.N;
+    int32_t *table = a.cell_table + (size_t)bh * a.cells;
+    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < a.N; j += gridDim.x * blockDim.x)
+        atomicAdd(table + code_cell(__ldg(codes + j), a.Ch, a.Cw), 1);
+}
+
+// one block per head: the non-empty cells in cell order -> (code, weight) items
+__global__ void __launch_bounds__(1024) dedupe_compact_kernel(SelectArgs a)
+{
+    __shared__ int wsum[32];
+    __shared__ int carry;
+    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t *table = a.cell_table + (size_t)bh * a.cells;
+    uint32_t *icode = a.item_code + (size_t)bh * a.N;
+    uint32_t *iw = a.item_weight + (size_t)bh * a.N;
+    if (tid == 0)
+        carry = 0;
+    __syncthreads();
+    for (int base = 0; base < a.cells; base += 1024) {
+        const int cell = base + tid;
+        const int n = cell < a.cells ? table[cell] : 0;
+        const uint32_t m = __ballot_sync(0xffffffffu, n > 0);
+        if (lane == 0)
+            wsum[warp] = __popc(m);
+        __syncthreads();
+        int before = carry;
+        for (int w = 0; w < warp; ++w)
+            before += wsum[w];
+        if (n > 0) {
+            const int slot = before + __popc(m & ((1u << lane) - 1u));
+            const int zw = cell % a.Cw, zh = (cell / a.Cw) % a.Ch, zt = cell / (a.Cw * a.Ch);
+            icode[slot] = (uint32_t)zt | ((uint32_t)zh << kCodeBits) | ((uint32_t)zw << (2 * kCodeBits));
+            iw[slot] = (uint32_t)n;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int tot = 0;
+            for (int w = 0; w < 32; ++w)
+                tot += wsum[w];
+            carry += tot;
+        }
+        __syncthreads();
+    }
+    if (tid == 0)
+        a.item_count[bh] = carry;
+}
+
+__global__ void __launch_bounds__(256) items_from_keys_kernel(SelectArgs a)
+{
+    const int bh = blockIdx.y;
+    const uint32_t *codes = a.codes + (size_t)bh * a.N;
+    uint32_t *icode = a.item_code + (size_t)bh * a.N;
+    uint32_t *iw = a.item_weight + (size_t)bh * a.N;
+    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < a.N; j += gridDim.x * blockDim.x) {
+        icode[j] = codes[j];
+        iw[j] = 1u;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        a.item_count[bh] = a.N;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Top-p count t_c (Eq. 7) for R query clusters of one head.
 __global__ void __launch_bounds__(NT, 2) select_topp_kernel(SelectArgs a)
 {
@@ -176,7 +252,9 @@ __global__ void __launch_bounds__(NT, 2) select_topp_kernel(SelectArgs a)
 
     const int bh = blockIdx.y, c0 = blockIdx.x * R;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t *codes = a.codes + (size_t)bh * a.N;
+    const uint32_t *icode = a.item_code + (size_t)bh * a.N;
+    const uint32_t *iw = a.item_weight + (size_t)bh * a.N;
+    const int nitems = a.item_count[bh];
     RowTables lrt[R];
     load_tables(a, bh, c0, lut, lrt);
     if (tid < R) {
@@ -193,8 +271,8 @@ __global__ void __launch_bounds__(NT, 2) select_topp_kernel(SelectArgs a)
 #pragma unroll
         for (int r = 0; r < R; ++r)
             m[r] = 0u;
-        for (int j = tid; j < a.N; j += NT) {
-            uint32_t code = __ldg(codes + j);
+        for (int i = tid; i < nitems; i += NT) {
+            uint32_t code = __ldg(icode + i);
 #pragma unroll
             for (int r = 0; r < R; ++r)
                 m[r] = max(m[r], order_key(proxy_raw(lrt[r], code)));
@@ -226,8 +304,9 @@ __global__ void __launch_bounds__(NT, 2) select_topp_kernel(SelectArgs a)
 #pragma unroll
         for (int r = 0; r < R; ++r)
             pf[r] = prefix[r];
-        for (int j = tid; j < a.N; j += NT) {
-            uint32_t code = __ldg(codes + j);
+        for (int i = tid; i < nitems; i += NT) {
+            const uint32_t code = __ldg(icode + i);
+            const uint32_t w = __ldg(iw + i);  // keys that share this composite code (and so this logit)
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 float raw = proxy_raw(lrt[r], code);
@@ -235,8 +314,8 @@ __global__ void __launch_bounds__(NT, 2) select_topp_kernel(SelectArgs a)
                 if (lv == 0 || (key >> pshift) == pf[r]) {
                     int bin = (key >> shift) & (nb - 1);
                     double e = exp((double)__fmul_rn(raw + 0.0f, a.scale) - mx[r]);
-                    atomicAdd(&cnt[r * NB + bin], 1u);
-                    atomicAdd(&mass[r * NB + bin], e);
+                    atomicAdd(&cnt[r * NB + bin], w);
+                    atomicAdd(&mass[r * NB + bin], (double)w * e);
                 }
             }
         }
@@ -408,6 +487,9 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
     const int bh = blockIdx.y, c0 = blockIdx.x * R;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t *codes = a.codes + (size_t)bh * a.N;
+    const uint32_t *icode = a.item_code + (size_t)bh * a.N;
+    const uint32_t *iw = a.item_weight + (size_t)bh * a.N;
+    const int nitems = a.item_count[bh];
     RowTables lrt[R];
     load_tables(a, bh, c0, lut, lrt);
     if (tid < R) {
@@ -457,15 +539,16 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
                 pf[r] = prefix[r];
                 td[r] = todo[r];
             }
-            for (int j = tid; j < a.N; j += NT) {
-                uint32_t code = __ldg(codes + j);
+            for (int i = tid; i < nitems; i += NT) {
+                const uint32_t code = __ldg(icode + i);
+                const uint32_t w = __ldg(iw + i);
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
                     if (!td[r])
                         continue;
                     uint32_t key = order_key(proxy_raw(lrt[r], code));
                     if (lv == 0 || (key >> pshift) == pf[r])
-                        atomicAdd(&cnt[r * NB + ((key >> shift) & (nb - 1))], 1u);
+                        atomicAdd(&cnt[r * NB + ((key >> shift) & (nb - 1))], w);
                 }
             }
             __syncthreads();
@@ -575,6 +658,14 @@ void launch_select(const SelectArgs &a, cudaStream_t st)
 {
     cudaFuncSetAttribute(select_topp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topp_smem(a));
     cudaFuncSetAttribute(select_emit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)emit_smem(a));
+    if (a.cells > 0) {
+        cudaMemsetAsync(a.cell_table, 0, (size_t)a.BH * a.cells * sizeof(int32_t), st);
+        dedupe_count_kernel<<<dim3(std::min(64, (a.N + 255) / 256), a.BH), 256, 0, st>>>(a);
+        dedupe_compact_kernel<<<a.BH, 1024, 0, st>>>(a);
+    } else {
+        items_from_keys_kernel<<<dim3(std::min(64, (a.N + 255) / 256), a.BH), 256, 0, st>>>(a);
+    }
+    count_launch(a.cells > 0 ? 2 : 1);
     dim3 grid((a.Cq + R - 1) / R, a.BH);
     select_topp_kernel<<<grid, NT, topp_smem(a), st>>>(a);
     khead_kernel<<<1, 1024, 0, st>>>(a);

@@ -353,3 +353,14 @@ def test_dense_mode_many_blocks():
         ref = orc.dense_rows(Q[0, h], K[0, h], V[0, h], cfg.scale, rows)
         err, rel = _attn_errors(Od[0, h][rows], ref)
         assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (h, err, rel)
+
+
+def test_large_code_space_without_count_table():
+    """C_T C_H C_W above the count-table limit: every key is its own item in the threshold searches."""
+    cfg = inputs.ScopeConfig("bigcodes", 1, 2, (5, 12, 12), (16, 56, 56), 24, 65, 65, 65, 3, 0.9, 48)
+    Q, K, V, dQ, dK, dV = _layer(cfg, 13)
+    ref = _oracle_plans(Q, K, cfg)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.H * cfg.Cq * cfg.N))
+    sb.scope_plan(dQ, dK, plan)
+    plan.check()
+    _compare_plan(plan, ref, cfg)
