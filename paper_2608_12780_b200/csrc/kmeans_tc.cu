@@ -2,15 +2,16 @@
 // of X), for codebooks that fit shared memory; kmeans.cu holds the general kernel.
 //
 // x.u for a tile of 128 tokens against every centroid is one tcgen05 MMA chain: A = the X tile
-// (bf16, exact), B = the centroids split into three bf16 terms u = hi + mid + lo (exact to 24
-// bits), all three chains accumulating into the same fp32 columns of tensor memory.  Each thread
+// (bf16, exact), B = the centroids split into two bf16 terms u = hi + lo (good to 2^-18 relative),
+// both chains accumulating into the same fp32 columns of tensor memory.  Each thread
 // then owns one token (one TMEM lane), forms |u|^2 - 2 x.u per centroid and keeps the two smallest.
 // As in the general kernel the label is final only if the gap between those two exceeds the
 // worst-case rounding error of this pass; otherwise the token is re-evaluated in fp64 with the
 // plain sum of squared differences.  Member sums are accumulated in fp64.
 //
-// A block holds the codebook splits once and runs two independent 128-thread pipelines (token
-// tiles alternate between them), so the loads / MMA of one overlap the epilogue of the other.
+// A block holds the codebook splits once and runs up to four independent 128-thread pipelines (token
+// tiles rotate over them), so the loads / MMA of one overlap the scalar work of the others; how many
+// fit is decided by shared memory and by the 512 columns of tensor memory.
 #include "scope_internal.cuh"
 #include "sm100.cuh"
 
@@ -21,11 +22,11 @@ using namespace sm100;
 namespace {
 
 constexpr int TM = 128;          // tokens per tile = MMA M
-constexpr int GROUPS = 2;        // independent pipelines per block
-constexpr int NT = 128 * GROUPS;
+constexpr int MAX_GROUPS = 4;    // independent pipelines per block
+constexpr int NSPLIT = 2;        // bf16 terms per centroid
+constexpr int NT = 128 * MAX_GROUPS;
 constexpr int HALF_BYTES = TM * 128;           // one 64-channel half of a 128-row tile
 constexpr int XTILE_BYTES = 2 * HALF_BYTES;    // 32 KB
-constexpr int TMEM_COLS_PER_GROUP = 256;
 
 struct TcLayout {
     int cpad[3];       // centroids padded to a multiple of 16
@@ -34,6 +35,7 @@ struct TcLayout {
     int un_off[3];     // float offset of the space's norms
     int cent_bytes;    // all split tiles
     int un_floats;
+    int cols;          // TMEM columns one pipeline needs (multiple of 32)
 };
 
 __host__ __device__ inline bool tc_layout(const KmArgs &a, TcLayout &L)
@@ -47,27 +49,28 @@ __host__ __device__ inline bool tc_layout(const KmArgs &a, TcLayout &L)
         L.col[s] = col;
         col += (cp + 31) & ~31;
         L.cent_off[s] = off;
-        off += 3 * 2 * cp * 128;  // 3 splits x 2 channel halves x cp rows x 128 B
+        off += NSPLIT * 2 * cp * 128;  // splits x 2 channel halves x cp rows x 128 B
         L.un_off[s] = un;
         un += cp;
     }
     L.cent_bytes = off;
     L.un_floats = un;
-    return col <= TMEM_COLS_PER_GROUP;
+    L.cols = col;
+    return col <= 256;
 }
 
 constexpr int MAXC = 256;  // centroids per range this kernel holds
 
 struct GroupShared {
-    int asg[3][TM];              // label of every token of the tile, per range
-    int pos[3][TM];              // slot of the token inside its label's run
+    uint16_t asg[3][TM];         // label of every token of the tile, per range
+    uint8_t pos[3][TM];          // slot of the token inside its label's run
     int cnt[3][MAXC];            // members per label in this tile
-    int start[3][MAXC];          // first slot of the label's run
+    uint8_t start[3][MAXC];      // first slot of the label's run
     uint32_t runs[3][TM];        // non-empty labels: label | start << 10 | count << 18
     int nruns[3];
     uint8_t sorted[3][TM];       // tokens of the tile grouped by label
     float x2[TM];                // squared norm of the token's row
-    int flagged[3 * TM];
+    uint16_t flagged[3 * TM];    // range << 8 | token
     int nflagged;
     int dead;
     uint64_t mbar;
@@ -85,7 +88,7 @@ __device__ __forceinline__ void load_x_tile(const KmArgs &a, const bf16 *Xh, int
     cp_async_commit();
 }
 
-__global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int tiles_per_block, int32_t *status)
+__global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int tiles_per_block, int groups, int32_t *status)
 {
     extern __shared__ unsigned char smem_dyn[];
     // 1024-byte alignment for the swizzled tiles
@@ -93,8 +96,8 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
     TcLayout L;
     tc_layout(a, L);
     unsigned char *s_cent = smem;
-    unsigned char *s_x = s_cent + L.cent_bytes;                       // GROUPS tiles
-    float *s_un = reinterpret_cast<float *>(s_x + GROUPS * XTILE_BYTES);
+    unsigned char *s_x = s_cent + L.cent_bytes;                       // one tile per pipeline
+    float *s_un = reinterpret_cast<float *>(s_x + groups * XTILE_BYTES);
     GroupShared *s_g = reinterpret_cast<GroupShared *>(s_un + ((L.un_floats + 3) & ~3));
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_timeout;
@@ -108,7 +111,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
     GroupShared &G = s_g[grp];
 
     if (warp == 0) {
-        tmem_alloc(&s_tmem_base, GROUPS * TMEM_COLS_PER_GROUP);
+        tmem_alloc(&s_tmem_base, 512);
         tmem_relinquish();
     }
     if (tid == 0)
@@ -121,18 +124,17 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
     // codebook splits and norms -> shared memory (once per block)
     for (int s = 0; s < a.nspaces; ++s) {
         const int cp = L.cpad[s];
-        const bf16 *src = a.sp[s].split + (size_t)bh * 3 * cp * kHeadDim;
-        const int nchunks = 3 * cp * 16;  // 16-byte chunks
-        for (int e = tid; e < nchunks; e += NT) {
+        const bf16 *src = a.sp[s].split + (size_t)bh * 3 * cp * kHeadDim;  // the first NSPLIT of the three stored terms
+        const int nchunks = NSPLIT * cp * 16;  // 16-byte chunks
+        for (int e = tid; e < nchunks; e += blockDim.x) {
             int chunk = e & 15, row = (e >> 4) % cp, p = (e >> 4) / cp;
             uint32_t dst = smem_u32(s_cent) + L.cent_off[s] + (p * 2 + (chunk >> 3)) * cp * 128 + sw128(row, chunk & 7);
             cp_async16(dst, src + ((size_t)p * cp + row) * kHeadDim + chunk * 8);
         }
-        for (int e = tid; e < cp; e += NT)
+        for (int e = tid; e < cp; e += blockDim.x)
             s_un[L.un_off[s] + e] = e < a.sp[s].C ? a.sp[s].unorm[(size_t)bh * a.sp[s].C + e] : INFINITY;
     }
     cp_async_commit();
-    const uint32_t tmem = s_tmem_base + grp * TMEM_COLS_PER_GROUP;  // read after the barrier below
     const uint32_t xbase = smem_u32(s_x) + grp * XTILE_BYTES;
     const int ntiles = (a.N + TM - 1) / TM;
     const int first = blockIdx.x * tiles_per_block + grp;
@@ -142,15 +144,14 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_g = *reinterpret_cast<volatile uint32_t *>(&s_tmem_base) + grp * TMEM_COLS_PER_GROUP;
-    (void)tmem;
+    const uint32_t tmem_g = *reinterpret_cast<volatile uint32_t *>(&s_tmem_base) + grp * L.cols;
     uint32_t phase = 0;
     bool dead = false;
     // descriptor words: high word fixed, low word = start address
     const uint64_t d0 = smem_desc_sw128(0);
     const uint32_t d_hi = (uint32_t)(d0 >> 32), d_lo = (uint32_t)d0;
 
-    for (int tile = first; tile < last && !dead; tile += GROUPS) {
+    for (int tile = first; tile < last && !dead; tile += groups) {
         const int tok0 = tile * TM;
         const bool valid = tok0 + gt < a.N;
         load_x_tile(a, Xh, tok0, xbase, gt);
@@ -168,7 +169,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                 const int k_lo = a.sp[s].ch0 >> 4, k_hi = (a.sp[s].ch0 + a.sp[s].D + 15) >> 4;
                 const uint32_t cb = smem_u32(s_cent) + L.cent_off[s];
                 bool acc = false;
-                for (int p = 0; p < 3; ++p)
+                for (int p = 0; p < NSPLIT; ++p)
                     for (int ks = k_lo; ks < k_hi; ++ks) {
                         const uint32_t ao = (xbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4;
                         const uint32_t bo = (cb + (p * 2 + (ks >> 2)) * cp * 128 + (ks & 3) * 32) >> 4;
@@ -246,16 +247,17 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                         }
                     }
                 }
-                G.asg[s][gt] = arg;
+                G.asg[s][gt] = (uint16_t)arg;
                 const int cbeg = a.sp[s].ch0 & ~15, cend = (a.sp[s].ch0 + a.sp[s].D + 15) & ~15;
-                // error budget of two tensor-core evaluations of |u|^2 - 2 x.u: the products are exact, each
-                // of the 3 * (channels / 16) accumulating MMAs may lose up to two fp32 ulps of the running
-                // magnitude (truncating adds), |x.u| <= (|u|^2 + |x|^2) / 2; doubled for margin
-                const float kappa = 8.f * (float)(3 * ((cend - cbeg) >> 4) + 2) * 1.1920929e-7f;
+                // error budget of two tensor-core evaluations of |u|^2 - 2 x.u: the products are exact, each of
+                // the NSPLIT * (channels / 16) accumulating MMAs may lose up to two fp32 ulps of the running
+                // magnitude (truncating adds), the two-term centroids are off by at most 2^-18 relative, and
+                // |x.u| <= (|u|^2 + |x|^2) / 2; doubled for margin
+                const float kappa = 8.f * (float)(NSPLIT * ((cend - cbeg) >> 4) + 2) * 1.1920929e-7f + 2.f * 3.8146973e-6f;
                 const float tol = kappa * (__ldg(a.sp[s].u2max + bh) + x2);
                 if (valid && C > 1 && second - best <= tol) {
                     int slot = atomicAdd(&G.nflagged, 1);
-                    G.flagged[slot] = (s << 16) | gt;
+                    G.flagged[slot] = (uint16_t)((s << 8) | gt);
                 }
             }
         }
@@ -271,7 +273,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         {
             const int nf = G.nflagged;
             for (int f = gw; f < nf; f += 4) {
-                const int s = G.flagged[f] >> 16, lt = G.flagged[f] & 0xffff;
+                const int s = G.flagged[f] >> 8, lt = G.flagged[f] & 0xff;
                 const KmSpace &sp = a.sp[s];
                 const float *cent = sp.cent + (size_t)bh * sp.C * sp.D;
                 const bf16 *x = Xh + (int64_t)(tok0 + lt) * a.sn + sp.ch0;
@@ -307,7 +309,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                     }
                 }
                 if (lane == 0)
-                    G.asg[s][lt] = ba;
+                    G.asg[s][lt] = (uint16_t)ba;
             }
         }
         bar_sync(1 + grp, 128);
@@ -317,7 +319,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         if (valid) {
             for (int s = 0; s < a.nspaces; ++s) {
                 lab[s] = G.asg[s][gt];
-                G.pos[s][gt] = atomicAdd(&G.cnt[s][lab[s]], 1);
+                G.pos[s][gt] = (uint8_t)atomicAdd(&G.cnt[s][lab[s]], 1);
             }
             if (a.nspaces == 1)
                 a.assign[(size_t)bh * a.N + tok0 + gt] = lab[0];
@@ -342,7 +344,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                 }
                 const int st = base + inc - n;
                 if (c < cp)
-                    G.start[s][c] = st;
+                    G.start[s][c] = (uint8_t)st;
                 const uint32_t m = __ballot_sync(0xffffffffu, n > 0);
                 if (n > 0)
                     G.runs[s][nr + __popc(m & ((1u << lane) - 1u))] = (uint32_t)c | ((uint32_t)st << 10) | ((uint32_t)n << 18);
@@ -401,40 +403,52 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
     tc_fence_before();
     __syncthreads();
     if (warp == 0)
-        tmem_dealloc(s_tmem_base, GROUPS * TMEM_COLS_PER_GROUP);
+        tmem_dealloc(s_tmem_base, 512);
     if (tid == 0 && s_timeout)
         atomicCAS(status + ST_CODE, 0, (int)SCOPE_ERR_TIMEOUT);
 }
 
 }  // namespace
 
-bool kmeans_tc_supported(const KmArgs &a, size_t *smem_bytes)
+// How many pipelines fit: shared memory (codebook splits once, one X tile and one scratch block per
+// pipeline) and the 512 tensor-memory columns of the SM.
+static int tc_groups(const KmArgs &a, size_t *smem_bytes)
 {
     TcLayout L;
     if (!tc_layout(a, L))
-        return false;
+        return 0;
     for (int s = 0; s < a.nspaces; ++s)
         if (!a.sp[s].split)
-            return false;
-    size_t need = 1024 + (size_t)L.cent_bytes + GROUPS * XTILE_BYTES + ((L.un_floats + 3) & ~3) * sizeof(float) +
-                  GROUPS * sizeof(GroupShared) + 64;
-    if (smem_bytes)
-        *smem_bytes = need;
-    return need <= 220 * 1024;
+            return 0;
+    for (int g = MAX_GROUPS; g >= 1; --g) {
+        size_t need = 1024 + (size_t)L.cent_bytes + (size_t)g * XTILE_BYTES + ((L.un_floats + 3) & ~3) * sizeof(float) +
+                      (size_t)g * sizeof(GroupShared) + 64;
+        if (need <= 226 * 1024 && g * L.cols <= 512) {
+            if (smem_bytes)
+                *smem_bytes = need;
+            return g;
+        }
+    }
+    return 0;
+}
+
+bool kmeans_tc_supported(const KmArgs &a, size_t *smem_bytes)
+{
+    return tc_groups(a, smem_bytes) >= 1;
 }
 
 void launch_kmeans_assign_tc(const KmArgs &a, int32_t *status, cudaStream_t st)
 {
     size_t smem = 0;
-    kmeans_tc_supported(a, &smem);
+    const int groups = tc_groups(a, &smem);
     // a block must own its SM (it allocates all 512 TMEM columns): ask for more than half the shared memory
     if (smem < 120 * 1024)
         smem = 120 * 1024;
     cudaFuncSetAttribute(kmeans_assign_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     const int ntiles = (a.N + TM - 1) / TM;
-    const int tiles_per_block = 8;
+    const int tiles_per_block = 4 * groups;
     dim3 grid((ntiles + tiles_per_block - 1) / tiles_per_block, a.B * a.H);
-    kmeans_assign_tc_kernel<<<grid, NT, smem, st>>>(a, tiles_per_block, status);
+    kmeans_assign_tc_kernel<<<grid, 128 * groups, smem, st>>>(a, tiles_per_block, groups, status);
     count_launch();
 }
 
