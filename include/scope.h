@@ -64,7 +64,14 @@ typedef struct {
     int64_t stride_b, stride_h, stride_n; /* elements; all 0 selects dense [B,H,N,d] */
     int64_t index_capacity;   /* entries the key-index buffer can hold, summed over all
                                  (batch, head, query cluster) */
+    int32_t select_mode;      /* SCOPE_SELECT_* below; 0 is the method of the paper */
+    int32_t reserved;         /* must be 0 */
 } scope_params;
+
+/* Key-count rules.  ONLINE is the paper's method (Eq. 8 - Eq. 10).  The other two are the variants
+ * its ablation compares against: FIXED stops after Eq. 8 (r_c = b_c, no per-head extension; k_head is
+ * still reported), TOPP keeps the Top-p count alone (b_c = r_c = t_c, k_fix unused). */
+enum { SCOPE_SELECT_ONLINE = 0, SCOPE_SELECT_FIXED = 1, SCOPE_SELECT_TOPP = 2 };
 
 typedef struct scope_plan_s scope_plan_t; /* opaque host object */
 

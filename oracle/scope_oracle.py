@@ -156,8 +156,12 @@ class HeadPlan:
     q_sse: np.ndarray  # query k-means SSE per iteration
 
 
-def select_head(P, z, n_c, N: int, scale: float, top_p: float, k_fix: int):
-    """Algorithm 3 given tables, codes and cluster sizes: (t_c, b_c, k_head, r_c, S, margin)."""
+def select_head(P, z, n_c, N: int, scale: float, top_p: float, k_fix: int, mode: str = "online"):
+    """Algorithm 3 given tables, codes and cluster sizes: (t_c, b_c, k_head, r_c, S, margin).
+
+    ``mode`` names the rule for the final counts: "online" is Algorithm 3 as printed; "fixed" is the
+    ablation's hybrid Top-p / fixed-Top-k without the per-head extension (r_c = b_c); "topp" is pure
+    Top-p (b_c = r_c = t_c)."""
     Cq = P[0].shape[0]
     orders, t = [], np.empty(Cq, np.int32)
     margin = np.inf
@@ -167,6 +171,14 @@ def select_head(P, z, n_c, N: int, scale: float, top_p: float, k_fix: int):
         orders.append(order)
         margin = min(margin, m)
     b, k, r = khead(n_c, t, N, k_fix)
+    if mode == "fixed":
+        r = b.copy()
+    elif mode == "topp":
+        b = t.copy()
+        k = -(-int((n_c.astype(np.int64) * b).sum()) // N)
+        r = t.copy()
+    else:
+        assert mode == "online"
     S = [key_set(orders[c], int(r[c])) for c in range(Cq)]
     return t, b, k, r, S, margin
 
@@ -183,7 +195,7 @@ def plan_head(Q, K, p) -> HeadPlan:
     ks = [kmeans(K, ch0, D, Cn, p.iters) for ch0, D, Cn in ranges]
     P = tuple(lut(kq.U, ch0, km.U)[0] for (ch0, _, _), km in zip(ranges, ks))
     z = tuple(km.assign for km in ks)
-    t, b, k, r, S, margin = select_head(P, z, kq.counts, N, p.scale, p.top_p, p.k_fix)
+    t, b, k, r, S, margin = select_head(P, z, kq.counts, N, p.scale, p.top_p, p.k_fix, getattr(p, "select_mode", "online"))
     gap = min(float(kq.min_gap.min()), *(float(km.min_gap.min()) for km in ks))
     return HeadPlan(kq.U, kq.assign, kq.counts, tuple(km.U for km in ks), z, P, t, b, k, r, S, gap, margin, kq.sse)
 

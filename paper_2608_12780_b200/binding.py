@@ -40,7 +40,7 @@ class ScopeParams(C.Structure):
                 ("Cq", C.c_int32), ("Ct", C.c_int32), ("Ch", C.c_int32), ("Cw", C.c_int32),
                 ("kmeans_iters", C.c_int32), ("top_p", C.c_float), ("k_fix", C.c_int32), ("scale", C.c_float),
                 ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_n", C.c_int64),
-                ("index_capacity", C.c_int64)]
+                ("index_capacity", C.c_int64), ("select_mode", C.c_int32), ("reserved", C.c_int32)]
 
 
 class ScopeError(RuntimeError):
@@ -112,7 +112,11 @@ def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 
 
-def make_params(cfg, B=None, H=None, index_capacity=None, strides=(0, 0, 0), scale=None) -> ScopeParams:
+SELECT_ONLINE, SELECT_FIXED, SELECT_TOPP = 0, 1, 2
+
+
+def make_params(cfg, B=None, H=None, index_capacity=None, strides=(0, 0, 0), scale=None,
+                select_mode=SELECT_ONLINE) -> ScopeParams:
     """ScopeParams from a config object with grid/split/Cq/... attributes (see inputs.ScopeConfig)."""
     B = cfg.B if B is None else B
     H = cfg.H if H is None else H
@@ -121,7 +125,7 @@ def make_params(cfg, B=None, H=None, index_capacity=None, strides=(0, 0, 0), sca
         index_capacity = max(1, int(0.35 * B * H * cfg.Cq * N))
     return ScopeParams(B, H, N, cfg.d, cfg.split[0], cfg.split[1], cfg.split[2], cfg.Cq, cfg.Ct, cfg.Ch, cfg.Cw,
                        cfg.iters, cfg.top_p, cfg.k_fix, cfg.scale if scale is None else scale,
-                       strides[0], strides[1], strides[2], int(index_capacity))
+                       strides[0], strides[1], strides[2], int(index_capacity), int(select_mode), 0)
 
 
 def _dev_ptr(t: torch.Tensor, name: str) -> int:

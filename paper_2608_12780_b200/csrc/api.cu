@@ -87,6 +87,8 @@ scope_status validate(const scope_params *p)
         return SCOPE_ERR_INVALID_ARG;
     if (p->index_capacity < 1)
         return SCOPE_ERR_INVALID_ARG;
+    if (p->select_mode < SCOPE_SELECT_ONLINE || p->select_mode > SCOPE_SELECT_TOPP || p->reserved != 0)
+        return SCOPE_ERR_INVALID_ARG;
     const bool dense = p->stride_b == 0 && p->stride_h == 0 && p->stride_n == 0;
     if (!dense) {
         if (p->stride_n < p->d || p->stride_h < 1 || p->stride_b < 1)
@@ -366,6 +368,7 @@ scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, u
         SelectArgs a{};
         a.BH = pl->BH; a.N = p.N; a.Cq = p.Cq; a.Ct = p.Ct; a.Ch = p.Ch; a.Cw = p.Cw;
         a.scale = p.scale; a.top_p = p.top_p; a.k_fix = p.k_fix; a.capacity = p.index_capacity;
+        a.select_mode = p.select_mode;
         a.codes = pl->k_codes;
         a.item_code = pl->item_code; a.item_weight = pl->item_weight; a.item_count = pl->item_count;
         a.cell_table = pl->cell_table; a.cells = pl->cells;

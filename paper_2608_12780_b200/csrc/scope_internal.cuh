@@ -54,6 +54,7 @@ struct SelectArgs {
     float scale;
     float top_p;
     int k_fix;
+    int select_mode;         // SCOPE_SELECT_*
     int64_t capacity;
     const uint32_t *codes;   // [BH, N]
     uint32_t *item_code;     // [BH, N] scratch: distinct composite codes of the head ...

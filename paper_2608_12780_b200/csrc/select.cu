@@ -393,7 +393,7 @@ __global__ void __launch_bounds__(1024) khead_kernel(SelectArgs a)
         unsigned long long num = 0;
         for (int c = tid; c < a.Cq; c += blockDim.x) {
             size_t row = (size_t)bh * a.Cq + c;
-            int b = max(a.t_c[row], a.k_fix);
+            int b = a.select_mode == SCOPE_SELECT_TOPP ? a.t_c[row] : max(a.t_c[row], a.k_fix);
             a.b_c[row] = b;
             num += (unsigned long long)a.n_c[row] * (unsigned long long)b;
         }
@@ -416,7 +416,7 @@ __global__ void __launch_bounds__(1024) khead_kernel(SelectArgs a)
             a.k_head[bh] = (int32_t)k;
         for (int c = tid; c < a.Cq; c += blockDim.x) {
             size_t row = (size_t)bh * a.Cq + c;
-            long long r = max((long long)a.b_c[row], k);
+            long long r = a.select_mode == SCOPE_SELECT_ONLINE ? max((long long)a.b_c[row], k) : (long long)a.b_c[row];
             a.r_c[row] = (int32_t)min(r, (long long)a.N);
         }
         __syncthreads();

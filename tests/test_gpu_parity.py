@@ -364,3 +364,20 @@ def test_large_code_space_without_count_table():
     sb.scope_plan(dQ, dK, plan)
     plan.check()
     _compare_plan(plan, ref, cfg)
+
+
+@pytest.mark.parametrize("mode,name", [(sb.SELECT_FIXED, "fixed"), (sb.SELECT_TOPP, "topp")])
+def test_selection_variants(mode, name):
+    cfg = inputs.CONFIGS["small"].replace(H=3)
+    Q, K, V, dQ, dK, dV = _layer(cfg, 14)
+    plan = sb.Plan(sb.make_params(cfg, select_mode=mode))
+    O = _to_np(sb.scope_forward(dQ, dK, dV, plan))
+    plan.check()
+    ocfg = cfg.replace()
+    object.__setattr__(ocfg, "select_mode", name)
+    ref = _oracle_plans(Q, K, ocfg)
+    _compare_plan(plan, ref, cfg)
+    for h in range(cfg.H):
+        Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], ref[h].g, ref[h].S, cfg.scale, np.arange(0, cfg.N, 3))
+        err, rel = _attn_errors(O[0, h][::3], Oref)
+        assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2

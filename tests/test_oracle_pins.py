@@ -384,3 +384,18 @@ def test_attention_uses_original_tokens_only():
         l = (k[S] @ q[i]) * float(np.float32(cfg.scale))
         w = np.exp(l - l.max())
         assert np.allclose(a[n], (w[:, None] * v[S]).sum(0) / w.sum(), rtol=0, atol=1e-6)
+
+
+def test_selection_variants_of_the_ablation():
+    cfg, Q, K, V = _head("tiny", seed=7)
+    pl = orc.plan_head(Q, K, cfg)
+    args = (pl.P, pl.z, pl.n_c, cfg.N, cfg.scale, cfg.top_p, cfg.k_fix)
+    t, b, k, r, S, _ = orc.select_head(*args, mode="online")
+    tf, bf, kf, rf, Sf, _ = orc.select_head(*args, mode="fixed")
+    tp, bp, kp, rp, Sp, _ = orc.select_head(*args, mode="topp")
+    assert np.array_equal(t, tf) and np.array_equal(t, tp)  # the Top-p counts do not depend on the rule
+    assert np.array_equal(bf, b) and np.array_equal(rf, b) and kf == k  # fixed: stops after Eq. 8
+    assert np.array_equal(bp, t) and np.array_equal(rp, t)  # pure Top-p
+    for c in range(cfg.Cq):  # nested along one ranking: pure Top-p <= fixed hybrid <= online
+        assert set(Sp[c].tolist()) <= set(Sf[c].tolist()) <= set(S[c].tolist())
+    assert (r > b).any()  # the online rule extends some cluster in this case
