@@ -156,6 +156,15 @@ scope_status scope_forward_host(const void *Q_host, const void *K_host, const vo
                                 scope_plan_t *plan, void *O_host, void *staging, size_t staging_bytes,
                                 void *stream);
 
+/* scope_forward_host without the final synchronisation: only enqueues the copies and the layer
+ * on `stream`.  O_host is valid, and errors found on the device are known, after the caller has
+ * synchronised the stream and called scope_plan_status().  Several plans (e.g. one per group of
+ * heads: heads are independent), each on its own stream with pinned host memory, overlap their
+ * copies with each other's kernels. */
+scope_status scope_forward_host_async(const void *Q_host, const void *K_host, const void *V_host,
+                                      scope_plan_t *plan, void *O_host, void *staging,
+                                      size_t staging_bytes, void *stream);
+
 /* Dense attention of Eq. 1 through the same attention kernel (every key selected,
  * identity query grouping); needs no plan arrays, only the plan's shape.  The
  * comparator of the benchmarks.  Asynchronous. */

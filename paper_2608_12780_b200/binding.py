@@ -28,7 +28,7 @@ STAGE_KMEANS_INIT, STAGE_KMEANS_Q, STAGE_KMEANS_K, STAGE_LUT, STAGE_SELECT, STAG
 STAGE_ALL = 63
 
 EXPORTS = ["scope_plan_workspace_bytes", "scope_plan_create", "scope_plan_destroy", "scope_plan", "scope_plan_stages",
-           "scope_sparse_attn", "scope_forward", "scope_forward_host", "scope_dense_attn", "scope_plan_status",
+           "scope_sparse_attn", "scope_forward", "scope_forward_host", "scope_forward_host_async", "scope_dense_attn", "scope_plan_status",
            "scope_plan_reset_status", "scope_plan_get", "scope_plan_field_bytes", "scope_plan_export",
            "scope_plan_import", "scope_status_string", "scope_kfix_from_alpha", "scope_kernel_launches",
            "scope_kmeans_queries_static"]
@@ -73,6 +73,7 @@ def lib():
         L.scope_dense_attn.argtypes = [vp, vp, vp, vp, vp, vp]
         L.scope_forward.argtypes = [vp, vp, vp, vp, vp, vp]
         L.scope_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+        L.scope_forward_host_async.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
         L.scope_plan_status.argtypes = [vp, vp, C.POINTER(i64)]
         L.scope_plan_reset_status.argtypes = [vp, vp]
         L.scope_plan_get.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(sz)]
@@ -258,15 +259,17 @@ def scope_forward(Q, K, V, plan: Plan, O=None):
     return O
 
 
-def scope_forward_host(Qh, Kh, Vh, plan: Plan, Oh, staging: torch.Tensor) -> None:
-    """The layer on HOST tensors (torch CPU bf16, ideally pinned); synchronous."""
+def scope_forward_host(Qh, Kh, Vh, plan: Plan, Oh, staging: torch.Tensor, sync: bool = True) -> None:
+    """The layer on HOST tensors (torch CPU bf16, ideally pinned).  With ``sync=False`` the call only
+    enqueues on the current stream (scope_forward_host_async): synchronise and ``plan.check()`` later."""
     for t in (Qh, Kh, Vh, Oh):
         if t.is_cuda or t.dtype != torch.bfloat16 or not t.is_contiguous():
             raise TypeError("host tensors must be contiguous CPU bfloat16")
     base = (staging.data_ptr() + 255) & ~255
     nbytes = staging.numel() * staging.element_size() - (base - staging.data_ptr())
-    _check(lib().scope_forward_host(Qh.data_ptr(), Kh.data_ptr(), Vh.data_ptr(), plan.handle, Oh.data_ptr(),
-                                    C.c_void_p(base), nbytes, C.c_void_p(_stream())), "scope_forward_host")
+    fn = lib().scope_forward_host if sync else lib().scope_forward_host_async
+    _check(fn(Qh.data_ptr(), Kh.data_ptr(), Vh.data_ptr(), plan.handle, Oh.data_ptr(),
+              C.c_void_p(base), nbytes, C.c_void_p(_stream())), "scope_forward_host")
 
 
 def scope_kmeans_queries_static(Q, C_clusters: int, iters: int):

@@ -429,8 +429,8 @@ scope_status scope_forward(const void *Q, const void *K, const void *V, scope_pl
     return scope_sparse_attn(Q, K, V, plan, O, stream);
 }
 
-scope_status scope_forward_host(const void *Qh, const void *Kh, const void *Vh, scope_plan_t *pl, void *Oh,
-                                void *staging, size_t staging_bytes, void *stream)
+static scope_status forward_host_enqueue(const void *Qh, const void *Kh, const void *Vh, scope_plan_t *pl, void *Oh,
+                                         void *staging, size_t staging_bytes, void *stream)
 {
     if (!pl || !Qh || !Kh || !Vh || !Oh || !staging)
         return SCOPE_ERR_INVALID_ARG;
@@ -454,7 +454,22 @@ scope_status scope_forward_host(const void *Qh, const void *Kh, const void *Vh, 
         return s;
     if (cudaMemcpyAsync(Oh, dO, one, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return SCOPE_ERR_CUDA;
+    return SCOPE_OK;
+}
+
+scope_status scope_forward_host(const void *Qh, const void *Kh, const void *Vh, scope_plan_t *pl, void *Oh,
+                                void *staging, size_t staging_bytes, void *stream)
+{
+    scope_status s = forward_host_enqueue(Qh, Kh, Vh, pl, Oh, staging, staging_bytes, stream);
+    if (s != SCOPE_OK)
+        return s;
     return scope_plan_status(pl, stream, nullptr);
+}
+
+scope_status scope_forward_host_async(const void *Qh, const void *Kh, const void *Vh, scope_plan_t *pl, void *Oh,
+                                      void *staging, size_t staging_bytes, void *stream)
+{
+    return forward_host_enqueue(Qh, Kh, Vh, pl, Oh, staging, staging_bytes, stream);
 }
 
 scope_status scope_plan_status(const scope_plan_t *pl, void *stream, int64_t *needed_capacity)

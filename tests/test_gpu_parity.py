@@ -381,3 +381,35 @@ def test_selection_variants(mode, name):
         Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], ref[h].g, ref[h].S, cfg.scale, np.arange(0, cfg.N, 3))
         err, rel = _attn_errors(O[0, h][::3], Oref)
         assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2
+
+
+def test_host_entry_points_match_device_path():
+    """scope_forward_host (and its asynchronous form on two head groups) against scope_forward."""
+    cfg = inputs.CONFIGS["small"]
+    Q, K, V, dQ, dK, dV = _layer(cfg, 15)
+    plan = sb.Plan(sb.make_params(cfg))
+    O_dev = sb.scope_forward(dQ, dK, dV, plan).cpu()
+    plan.check()
+    hQ, hK, hV = (sb.bits_to_torch(x, pin=True) for x in (Q, K, V))
+    hO = torch.empty_like(hQ).pin_memory()
+    nbytes = hQ.numel() * 2
+    staging = torch.empty(4 * nbytes + 512, dtype=torch.uint8, device="cuda")
+    sb.scope_forward_host(hQ, hK, hV, plan, hO, staging)
+    assert torch.equal(hO, O_dev)
+    with pytest.raises(sb.ScopeError):  # staging too small
+        sb.scope_forward_host(hQ, hK, hV, plan, hO, staging[: nbytes])
+    # two head groups on two streams
+    hO2 = torch.zeros_like(hO)
+    G, hg = 2, cfg.H // 2
+    plans = [sb.Plan(sb.make_params(cfg, H=hg)) for _ in range(G)]
+    stg = [torch.empty(4 * nbytes // G + 512, dtype=torch.uint8, device="cuda") for _ in range(G)]
+    streams = [torch.cuda.Stream() for _ in range(G)]
+    torch.cuda.synchronize()
+    for g in range(G):
+        with torch.cuda.stream(streams[g]):
+            sl = slice(g * hg, (g + 1) * hg)
+            sb.scope_forward_host(hQ[:, sl], hK[:, sl], hV[:, sl], plans[g], hO2[:, sl], stg[g], sync=False)
+    for g in range(G):
+        streams[g].synchronize()
+        plans[g].check()
+    assert torch.equal(hO2, O_dev)
