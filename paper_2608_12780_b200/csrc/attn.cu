@@ -198,7 +198,7 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
         };
         // LA tiles are in flight ahead of the one being handed over; tile t is handed over before
         // the slot for tile t + LA is waited for (that slot is freed by work that needs tile t)
-        constexpr int LA = STAGES - 1;
+        constexpr int LA = STAGES - 2;
         for (int i = 0; i < LA && i < ntiles; ++i) {
             load_idx(i);
             issue_tile(i % STAGES);
