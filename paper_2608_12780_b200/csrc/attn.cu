@@ -45,7 +45,7 @@ struct Barriers {
     uint64_t kv_full[STAGES];
     uint64_t kv_empty[STAGES];
     uint64_t s_full[QT][2];
-    uint64_t p_full[QT];
+    uint64_t p_full[QT][2];  // per S buffer, like s_full: a waiter can never fall two phases behind
     uint64_t pv_done[QT];
 };
 
@@ -152,7 +152,8 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
         for (int i = 0; i < QT; ++i) {
             mbar_init(&bars.s_full[i][0], 1);
             mbar_init(&bars.s_full[i][1], 1);
-            mbar_init(&bars.p_full[i], BM);
+            mbar_init(&bars.p_full[i][0], BM);
+            mbar_init(&bars.p_full[i][1], BM);
             mbar_init(&bars.pv_done[i], 1);
         }
         mbar_fence_init();
@@ -270,7 +271,7 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
                     tc_fence_after();
                     issue_s(t + 1);
                 }
-                alive = wait(&bars.p_full[i], (uint32_t)(t & 1), abort_flag);
+                alive = wait(&bars.p_full[i][t & 1], (uint32_t)((t >> 1) & 1), abort_flag);
                 if (!alive)
                     break;
                 tc_fence_after();
@@ -379,7 +380,7 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
             tmem_st32(sa, p);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(&bars.p_full[qt]);
+            mbar_arrive(&bars.p_full[qt][t & 1]);
         }
         // A parity wait is only meaningful one phase back.  Waits on pv_done are skipped whenever no
         // rescale is needed, so catch up one phase at a time: S of the last tile being complete implies
