@@ -29,6 +29,7 @@ struct scope_plan_s {
     int32_t *q_perm, *q_offsets;
     // scratch
     float *q_unorm, *k_unorm[3], *q_u2max, *k_u2max[3];
+    float *q_x2, *k_x2;  // squared row norms of Q and K, written by the first k-means pass of a call
     bf16 *q_split, *k_split[3];
     double *q_sums, *k_sums[3];
     int32_t *q_counts, *k_counts[3];
@@ -124,6 +125,8 @@ void carve(scope_plan_t *pl, unsigned char *base, size_t *total)
         pl->lut[m] = cv.take<float>(BH * Cq * C[m]);
     }
     pl->q_assign = cv.take<int32_t>(BH * N);
+    pl->q_x2 = cv.take<float>(BH * N);
+    pl->k_x2 = cv.take<float>(BH * N);
     pl->k_codes = cv.take<uint32_t>(BH * N);
     pl->n_c = cv.take<int32_t>(BH * Cq);
     pl->t_c = cv.take<int32_t>(BH * Cq);
@@ -174,6 +177,7 @@ KmArgs q_args(const scope_plan_t *pl, const void *Q)
                       pl->q_split, (p.Cq + 15) & ~15};
     a.assign = pl->q_assign;
     a.codes = nullptr;
+    a.x2 = pl->q_x2;
     return a;
 }
 
@@ -191,6 +195,7 @@ KmArgs k_args(const scope_plan_t *pl, const void *K)
                           pl->k_counts[m], nullptr, pl->k_split[m], (C[m] + 15) & ~15};
     a.assign = nullptr;
     a.codes = pl->k_codes;
+    a.x2 = pl->k_x2;
     return a;
 }
 
@@ -350,15 +355,19 @@ scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, u
         KmArgs a = q_args(pl, Q);
         if (!(stages & SCOPE_STAGE_KMEANS_INIT))
             launch_kmeans_norms(a, st);  // centroids may have been imported
-        for (int it = 0; it < p.kmeans_iters; ++it)
+        for (int it = 0; it < p.kmeans_iters; ++it) {
+            a.x2_ready = it > 0;
             launch_kmeans_iteration(a, pl->status, st);
+        }
     }
     if (stages & SCOPE_STAGE_KMEANS_K) {
         KmArgs a = k_args(pl, K);
         if (!(stages & SCOPE_STAGE_KMEANS_INIT))
             launch_kmeans_norms(a, st);
-        for (int it = 0; it < p.kmeans_iters; ++it)
+        for (int it = 0; it < p.kmeans_iters; ++it) {
+            a.x2_ready = it > 0;
             launch_kmeans_iteration(a, pl->status, st);
+        }
     }
     if (stages & SCOPE_STAGE_LUT) {
         KmArgs a = k_args(pl, K);

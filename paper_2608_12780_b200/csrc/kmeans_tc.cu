@@ -60,30 +60,38 @@ __host__ __device__ inline bool tc_layout(const KmArgs &a, TcLayout &L)
 }
 
 constexpr int MAXC = 256;  // centroids per range this kernel holds
+constexpr int MAXCAND = 128;  // (token, contender) pairs re-evaluated by one thread each, per tile
 
 struct GroupShared {
     uint16_t asg[3][TM];         // label of every token of the tile, per range
-    uint8_t pos[3][TM];          // slot of the token inside its label's run
-    int cnt[3][MAXC];            // members per label in this tile
+    uint32_t cnt[3][MAXC / 4];   // members per label in this tile, four 8-bit counters per word (a tile has 128 tokens)
     uint8_t start[3][MAXC];      // first slot of the label's run
     uint32_t runs[3][TM];        // non-empty labels: label | start << 10 | count << 18
     int nruns[3];
-    uint8_t sorted[3][TM];       // tokens of the tile grouped by label
-    float x2[TM];                // squared norm of the token's row
-    uint16_t flagged[3 * TM];    // range << 8 | token
+    uint16_t sorted[3][TM];      // tokens of the tile grouped by label, as the row part of their shared-memory address
+    uint16_t flagged[3 * TM];    // range << 8 | token: close calls that are re-evaluated against every centroid
     int nflagged;
+    uint32_t cand[MAXCAND];      // close calls with at most four contenders: centroid | token << 8 | range << 15 | k << 17 | n << 19
+    double cdist[MAXCAND];       // fp64 distance of each contender
+    int ncand;
     int dead;
     uint64_t mbar;
 };
 
 __device__ __forceinline__ void load_x_tile(const KmArgs &a, const bf16 *Xh, int tok0, uint32_t xbase, int gt)
 {
-    // 128 rows x 16 chunks of 16 bytes; rows past N are zero
-    for (int e = gt; e < TM * 16; e += 128) {
-        int row = e >> 4, chunk = e & 15;
-        bool ok = tok0 + row < a.N;
-        const bf16 *src = Xh + (int64_t)(ok ? tok0 + row : 0) * a.sn + chunk * 8;
-        cp_async16_zfill(xbase + (chunk >> 3) * HALF_BYTES + sw128(row, chunk & 7), src, ok ? 16 : 0);
+    // 128 rows x 16 chunks of 16 bytes; rows past N are zero.  A thread keeps its chunk and walks rows
+    // gt/16 + 8 i: the swizzle term depends on row & 7 only, so the destination advances by 1024 bytes.
+    const int row0 = gt >> 4, chunk = gt & 15;
+    const uint32_t dst = xbase + (chunk >> 3) * HALF_BYTES + sw128(row0, chunk & 7);
+    const bf16 *src = Xh + (int64_t)(tok0 + row0) * a.sn + chunk * 8;
+    const int64_t step = 8 * a.sn;
+    const int rows_left = a.N - tok0 - row0;  // row row0 + 8 i exists iff 8 i < rows_left
+#pragma unroll
+    for (int i = 0; i < TM / 8; ++i) {
+        const bool ok = 8 * i < rows_left;
+        cp_async16_zfill(dst + 1024 * i, ok ? src : Xh, ok ? 16 : 0);
+        src += step;
     }
     cp_async_commit();
 }
@@ -163,6 +171,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         if (gt == 0) {
             tc_fence_after();
             G.nflagged = 0;
+            G.ncand = 0;
             for (int s = 0; s < a.nspaces; ++s) {
                 const int cp = L.cpad[s];
                 const uint32_t idesc = idesc_bf16(TM, cp, false, false);
@@ -179,10 +188,15 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             }
             mma_commit(&G.mbar);
         }
-        for (int e = gt; e < a.nspaces * MAXC; e += 128)
-            (&G.cnt[0][0])[e] = 0;
-        {
-            // squared norm of the whole row (an upper bound of every range's slice, used in the tolerance)
+        for (int e = gt; e < a.nspaces * (MAXC / 4); e += 128)
+            (&G.cnt[0][0])[e] = 0u;
+        // squared norm of the whole row (an upper bound of every range's slice, used in the tolerance): taken
+        // from the tile in the first pass of a call and kept in global memory for the later ones
+        float x2 = 0.f;
+        if (a.x2 != nullptr && a.x2_ready) {
+            if (valid)
+                x2 = __ldg(a.x2 + (size_t)bh * a.N + tok0 + gt);
+        } else {
             float x2a = 0.f, x2b = 0.f;
 #pragma unroll
             for (int chunk = 0; chunk < 16; ++chunk) {
@@ -195,7 +209,9 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                     x2b = fmaf(hi, hi, x2b);
                 }
             }
-            G.x2[gt] = x2a + x2b;
+            x2 = x2a + x2b;
+            if (a.x2 != nullptr && valid)
+                a.x2[(size_t)bh * a.N + tok0 + gt] = x2;
         }
         // a wait that runs out is recorded and ends this pipeline after the next barrier
         const bool ok = __all_sync(0xffffffffu, mbar_wait(&G.mbar, phase));
@@ -206,7 +222,6 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         phase ^= 1;
         tc_fence_after();
         if (ok) {
-            const float x2 = G.x2[gt];
             for (int s = 0; s < a.nspaces; ++s) {
                 const int C = a.sp[s].C, cp = L.cpad[s];
                 const float *un = s_un + L.un_off[s];
@@ -255,9 +270,56 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                 // |x.u| <= (|u|^2 + |x|^2) / 2; doubled for margin
                 const float kappa = 8.f * (float)(NSPLIT * ((cend - cbeg) >> 4) + 2) * 1.1920929e-7f + 2.f * 3.8146973e-6f;
                 const float tol = kappa * (__ldg(a.sp[s].u2max + bh) + x2);
-                if (valid && C > 1 && second - best <= tol) {
-                    int slot = atomicAdd(&G.nflagged, 1);
-                    G.flagged[slot] = (uint16_t)((s << 8) | gt);
+                const bool close = valid && C > 1 && second - best <= tol;
+                if (__any_sync(0xffffffffu, close)) {
+                    // The true nearest centroid of a close call is among those whose distance in this pass is
+                    // within the budget of the best one: list them (second look at the row; the loads are
+                    // warp-wide, so the whole warp walks it).  Usually two.
+                    const float lim = best + tol;
+                    int nc = 0;
+                    uint32_t packed = 0;
+                    for (int c0 = 0; c0 < cp; c0 += 32) {
+                        uint32_t r[32];
+                        if (cp - c0 >= 32) {
+                            tmem_ld32(ta + c0, r);
+                        } else {
+                            uint32_t r16[16];
+                            tmem_ld16(ta + c0, r16);
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                r[j] = r16[j];
+                                r[16 + j] = 0u;
+                            }
+                        }
+                        tmem_wait_ld();
+                        const int nc32 = min(32, cp - c0);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (j < nc32) {
+                                const float dist = fmaf(-2.f, __uint_as_float(r[j]), un[c0 + j]);
+                                if (close && dist <= lim) {
+                                    if (nc < 4)
+                                        packed |= (uint32_t)(c0 + j) << (8 * nc);
+                                    ++nc;
+                                }
+                            }
+                        }
+                    }
+                    if (close) {
+                        int base = MAXCAND;
+                        if (nc <= 4)
+                            base = atomicAdd(&G.ncand, nc);
+                        if (base + nc <= MAXCAND) {
+                            for (int k = 0; k < nc; ++k)
+                                G.cand[base + k] = ((packed >> (8 * k)) & 0xffu) | ((uint32_t)gt << 8) | ((uint32_t)s << 15) |
+                                                   ((uint32_t)k << 17) | ((uint32_t)nc << 19);
+                        } else {  // many contenders (or a full list): every centroid is re-evaluated
+                            for (int k = base; k < MAXCAND; ++k)
+                                G.cand[k] = 1u << 17;  // reserved but unused slots: never the first of a token
+                            int slot = atomicAdd(&G.nflagged, 1);
+                            G.flagged[slot] = (uint16_t)((s << 8) | gt);
+                        }
+                    }
                 }
             }
         }
@@ -271,6 +333,41 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         // Every centroid's distance is summed in the same fixed order, so equal centroids tie exactly and
         // the lowest index wins, as in a plain sequential evaluation.
         {
+            // contenders: one thread each, channels in order (the fp64 sum must be the plain sequential one)
+            const int ncand = min(G.ncand, MAXCAND);  // entries past the list went to the full re-evaluation
+            if (ncand > 0) {
+                if (gt < ncand) {
+                    const uint32_t e = G.cand[gt];
+                    const int c = e & 0xff, lt = (e >> 8) & 0x7f, s = (e >> 15) & 3;
+                    const KmSpace &sp = a.sp[s];
+                    const float *u = sp.cent + ((size_t)bh * sp.C + c) * sp.D;
+                    double d = 0.0;
+#pragma unroll 8
+                    for (int ch = 0; ch < sp.D; ++ch) {
+                        const int ac = sp.ch0 + ch;
+                        const bf16 xb = *reinterpret_cast<const bf16 *>(s_x + grp * XTILE_BYTES + (ac >> 6) * HALF_BYTES +
+                                                                        sw128(lt, (ac & 63) >> 3) + (ac & 7) * 2);
+                        const double df = __dsub_rn((double)__bfloat162float(xb), (double)__ldg(u + ch));
+                        d = __dadd_rn(d, __dmul_rn(df, df));
+                    }
+                    G.cdist[gt] = d;
+                }
+                bar_sync(1 + grp, 128);
+                if (gt < ncand) {
+                    const uint32_t e = G.cand[gt];
+                    if (((e >> 17) & 3) == 0) {  // first contender of its token: ascending centroid order, lowest wins ties
+                        const int n = (e >> 19) & 7, lt = (e >> 8) & 0x7f, s = (e >> 15) & 3;
+                        double bd = G.cdist[gt];
+                        int ba = e & 0xff;
+                        for (int k = 1; k < n; ++k)
+                            if (G.cdist[gt + k] < bd) {
+                                bd = G.cdist[gt + k];
+                                ba = G.cand[gt + k] & 0xff;
+                            }
+                        G.asg[s][lt] = (uint16_t)ba;
+                    }
+                }
+            }
             const int nf = G.nflagged;
             for (int f = gw; f < nf; f += 4) {
                 const int s = G.flagged[f] >> 8, lt = G.flagged[f] & 0xff;
@@ -315,11 +412,12 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         bar_sync(1 + grp, 128);
 
         // ---- labels out, and the tile's tokens grouped by label (counting sort in shared memory)
-        int lab[3] = {0, 0, 0};
+        int lab[3] = {0, 0, 0}, pos[3] = {0, 0, 0};
         if (valid) {
             for (int s = 0; s < a.nspaces; ++s) {
                 lab[s] = G.asg[s][gt];
-                G.pos[s][gt] = (uint8_t)atomicAdd(&G.cnt[s][lab[s]], 1);
+                const int sh = (lab[s] & 3) * 8;
+                pos[s] = (int)((atomicAdd(&G.cnt[s][lab[s] >> 2], 1u << sh) >> sh) & 0xffu);
             }
             if (a.nspaces == 1)
                 a.assign[(size_t)bh * a.N + tok0 + gt] = lab[0];
@@ -334,7 +432,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             int base = 0, nr = 0;
             for (int c0 = 0; c0 < cp; c0 += 32) {
                 const int c = c0 + lane;
-                const int n = c < cp ? G.cnt[s][c] : 0;
+                const int n = c < cp ? (int)((G.cnt[s][c >> 2] >> ((c & 3) * 8)) & 0xffu) : 0;
                 int inc = n;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -357,40 +455,48 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         bar_sync(1 + grp, 128);
         if (valid)
             for (int s = 0; s < a.nspaces; ++s)
-                G.sorted[s][G.start[s][lab[s]] + G.pos[s][gt]] = (uint8_t)gt;
+                G.sorted[s][G.start[s][lab[s]] + pos[s]] = (uint16_t)sw128(gt, 0);
         bar_sync(1 + grp, 128);
 
-        // ---- member sums: one thread per channel, one fp64 atomic per (label present in the tile, channel)
+        // ---- member sums: a thread owns two adjacent channels (one 32-bit word of every row) and every other
+        // run of their range; one fp64 atomic per (label present in the tile, channel)
         {
-            const int ch = gt;
+            const int ch = 2 * (gt & 63), hf = gt >> 6;
             int s = 0;
             while (s + 1 < a.nspaces && ch >= a.sp[s].ch0 + a.sp[s].D)
                 ++s;
             const KmSpace &sp = a.sp[s];
             const int rel = ch - sp.ch0;
-            double *sums = sp.sums + (size_t)bh * sp.C * sp.D;
+            double *sums = sp.sums + (size_t)bh * sp.C * sp.D + rel;
             int32_t *counts = sp.counts + (size_t)bh * sp.C;
-            const unsigned char *xcol = s_x + grp * XTILE_BYTES + (ch >> 6) * HALF_BYTES + (ch & 7) * 2;
-            const int chunk = (ch & 63) >> 3;
+            // sw128(row, chunk) = sw128(row, 0) ^ (chunk << 4): the sorted list holds the row part
+            const uint32_t xpair = xbase + (ch >> 6) * HALF_BYTES + (ch & 7) * 2;
+            const uint32_t cbits = (uint32_t)((ch & 63) >> 3) << 4;
             const int nr = G.nruns[s];
-            for (int r = 0; r < nr; ++r) {
+            for (int r = hf; r < nr; r += 2) {
                 const uint32_t run = G.runs[s][r];
                 const int cl = run & 1023, st = (run >> 10) & 255, n = run >> 18;
-                const uint8_t *tok = &G.sorted[s][st];
-                double acc0 = 0.0, acc1 = 0.0;
+                const uint16_t *tok = &G.sorted[s][st];
+                // bf16 values of any magnitudes do not add exactly in fp32; in fp64 they do
+                double lo0 = 0.0, lo1 = 0.0, hi0 = 0.0, hi1 = 0.0;
                 int l = 0;
-                for (; l + 8 <= n; l += 8) {
-                    float v[8];
+                for (; l + 4 <= n; l += 4) {
+                    uint32_t w[4];
 #pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        v[q] = __bfloat162float(*reinterpret_cast<const bf16 *>(xcol + sw128(tok[l + q], chunk)));
-                    // bf16 values of any magnitudes do not add exactly in fp32; in fp64 they do
-                    acc0 += (((double)v[0] + (double)v[1]) + ((double)v[2] + (double)v[3]));
-                    acc1 += (((double)v[4] + (double)v[5]) + ((double)v[6] + (double)v[7]));
+                    for (int q = 0; q < 4; ++q)
+                        w[q] = lds32(xpair + ((uint32_t)tok[l + q] ^ cbits));
+                    lo0 += (double)__uint_as_float(w[0] << 16) + (double)__uint_as_float(w[1] << 16);
+                    hi0 += (double)__uint_as_float(w[0] & 0xffff0000u) + (double)__uint_as_float(w[1] & 0xffff0000u);
+                    lo1 += (double)__uint_as_float(w[2] << 16) + (double)__uint_as_float(w[3] << 16);
+                    hi1 += (double)__uint_as_float(w[2] & 0xffff0000u) + (double)__uint_as_float(w[3] & 0xffff0000u);
                 }
-                for (; l < n; ++l)
-                    acc0 += (double)__bfloat162float(*reinterpret_cast<const bf16 *>(xcol + sw128(tok[l], chunk)));
-                atomicAdd(sums + (size_t)cl * sp.D + rel, acc0 + acc1);
+                for (; l < n; ++l) {
+                    const uint32_t w = lds32(xpair + ((uint32_t)tok[l] ^ cbits));
+                    lo0 += (double)__uint_as_float(w << 16);
+                    hi0 += (double)__uint_as_float(w & 0xffff0000u);
+                }
+                atomicAdd(sums + (size_t)cl * sp.D, lo0 + lo1);
+                atomicAdd(sums + (size_t)cl * sp.D + 1, hi0 + hi1);
                 if (rel == 0)
                     atomicAdd(counts + cl, n);
             }

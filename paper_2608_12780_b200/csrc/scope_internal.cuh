@@ -41,6 +41,8 @@ struct KmArgs {
     KmSpace sp[3];
     int32_t *assign;   // [BH, N] labels (nspaces == 1)
     uint32_t *codes;   // [BH, N] packed labels (nspaces == 3)
+    float *x2;         // [BH, N] squared row norms, kept from the first pass to the later ones (may be null)
+    int x2_ready;      // 0: this pass computes and stores them, 1: it reads them
 };
 
 // Per (head, query cluster) result of the selection stage that later kernels read.

@@ -237,6 +237,14 @@ __device__ __forceinline__ void mma_ts2(uint32_t tmem_d, uint32_t tmem_a, uint32
         : "memory");
 }
 
+// 32-bit load from a shared-memory address given as a number (the swizzled tile addresses are computed, not indexed)
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
 // byte offset of 16-byte chunk `chunk` (0..7) of row `row` in a 128-byte-swizzled tile
 __device__ __forceinline__ uint32_t sw128(int row, int chunk)
 {
