@@ -74,6 +74,7 @@ struct GroupShared {
     uint32_t cand[MAXCAND];      // close calls with at most four contenders: centroid | token << 8 | range << 15 | k << 17 | n << 19
     double cdist[MAXCAND];       // fp64 distance of each contender
     int ncand;
+    int next_tile;               // the tile this pipeline takes after the current one
     int dead;
     uint64_t mbar;
 };
@@ -109,6 +110,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
     GroupShared *s_g = reinterpret_cast<GroupShared *>(s_un + ((L.un_floats + 3) & ~3));
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_timeout;
+    __shared__ int s_queue;  // next tile of the block's range nobody has taken yet
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int grp = tid >> 7, gt = tid & 127;       // pipeline, thread within it
@@ -122,8 +124,10 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         tmem_alloc(&s_tmem_base, 512);
         tmem_relinquish();
     }
-    if (tid == 0)
+    if (tid == 0) {
         s_timeout = 0;
+        s_queue = blockIdx.x * tiles_per_block + groups;  // the first `groups` tiles are taken by construction
+    }
     if (gt == 0) {
         G.dead = 0;
         mbar_init(&G.mbar, 1);
@@ -159,7 +163,8 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
     const uint64_t d0 = smem_desc_sw128(0);
     const uint32_t d_hi = (uint32_t)(d0 >> 32), d_lo = (uint32_t)d0;
 
-    for (int tile = first; tile < last && !dead; tile += groups) {
+    // the pipelines of a block share one queue over the block's tiles: whichever is free takes the next tile
+    for (int tile = first; tile < last && !dead; tile = G.next_tile) {
         const int tok0 = tile * TM;
         const bool valid = tok0 + gt < a.N;
         load_x_tile(a, Xh, tok0, xbase, gt);
@@ -226,8 +231,11 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                 const int C = a.sp[s].C, cp = L.cpad[s];
                 const float *un = s_un + L.un_off[s];
                 const uint32_t ta = tmem_g + ((uint32_t)(gw * 32) << 16) + L.col[s];
-                float best = INFINITY, second = INFINITY;
-                int arg = 0;
+                // four independent running (best, second, index) triples over the columns j % 4, merged at the
+                // end: the chain of dependent compares is what this loop waits on.  Which of several equal
+                // distances wins here does not matter: a zero gap is always a close call.
+                float bq[4] = {INFINITY, INFINITY, INFINITY, INFINITY}, sq[4] = {INFINITY, INFINITY, INFINITY, INFINITY};
+                int aq[4] = {0, 0, 0, 0};
                 for (int c0 = 0; c0 < cp; c0 += 32) {
                     uint32_t r[32];
                     if (cp - c0 >= 32) {
@@ -251,16 +259,20 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 const float dist = fmaf(-2.f, __uint_as_float(r[j4 + q]), uu[q]);
-                                if (dist < best) {
-                                    second = best;
-                                    best = dist;
-                                    arg = c0 + j4 + q;
-                                } else if (dist < second) {
-                                    second = dist;
-                                }
+                                sq[q] = fminf(sq[q], fmaxf(bq[q], dist));
+                                aq[q] = dist < bq[q] ? c0 + j4 + q : aq[q];
+                                bq[q] = fminf(bq[q], dist);
                             }
                         }
                     }
+                }
+                float best = bq[0], second = sq[0];
+                int arg = aq[0];
+#pragma unroll
+                for (int q = 1; q < 4; ++q) {
+                    second = fminf(fminf(second, sq[q]), fmaxf(best, bq[q]));
+                    arg = bq[q] < best ? aq[q] : arg;
+                    best = fminf(best, bq[q]);
                 }
                 G.asg[s][gt] = (uint16_t)arg;
                 const int cbeg = a.sp[s].ch0 & ~15, cend = (a.sp[s].ch0 + a.sp[s].D + 15) & ~15;
@@ -501,6 +513,8 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                     atomicAdd(counts + cl, n);
             }
         }
+        if (gt == 0)
+            G.next_tile = atomicAdd(&s_queue, 1);
         tc_fence_before();
         bar_sync(1 + grp, 128);  // the X tile and the label arrays are reused by the next tile
     }
@@ -552,8 +566,33 @@ void launch_kmeans_assign_tc(const KmArgs &a, int32_t *status, cudaStream_t st)
         smem = 120 * 1024;
     cudaFuncSetAttribute(kmeans_assign_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     const int ntiles = (a.N + TM - 1) / TM;
-    const int tiles_per_block = 4 * groups;
-    dim3 grid((ntiles + tiles_per_block - 1) / tiles_per_block, a.B * a.H);
+    // Blocks per head: a block pays for loading the codebook and ends when its slowest pipeline does, so few
+    // large blocks are better, as long as the grid fills whole waves of SMs.  Cost model: waves x (rounds of
+    // `groups` tiles per block + 2 rounds of fixed cost); ties go to more blocks.
+    static int num_sms = 0;
+    if (num_sms == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
+            num_sms = 148;
+    }
+    const int heads = a.B * a.H;
+    int best_bph = 1;
+    double best_cost = 1e300;
+    for (int bph = 1; bph <= (ntiles + groups - 1) / groups; ++bph) {
+        const int tpb = (ntiles + bph - 1) / bph;
+        const int nblk = (ntiles + tpb - 1) / tpb;  // blocks that get any tile
+        const double waves = (double)(((int64_t)heads * nblk + num_sms - 1) / num_sms);
+        const double cost = waves * ((tpb + groups - 1) / groups + 2.0);
+        if (cost <= best_cost) {
+            best_cost = cost;
+            best_bph = nblk;
+        }
+        if (tpb <= groups)
+            break;
+    }
+    const int tiles_per_block = (ntiles + best_bph - 1) / best_bph;
+    dim3 grid((ntiles + tiles_per_block - 1) / tiles_per_block, heads);
     kmeans_assign_tc_kernel<<<grid, 128 * groups, smem, st>>>(a, tiles_per_block, groups, status);
     count_launch();
 }
