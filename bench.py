@@ -380,7 +380,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="scope", choices=["scope", "reference"])
-    ap.add_argument("--workload", default="HY720", choices=sorted(inputs.CONFIGS))
+    ap.add_argument("--workload", default="HY720", choices=sorted(inputs.CONFIGS) + sorted(inputs.PAPER_SCALE_CONFIGS))
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--gen-threads", type=int, default=min(16, os.cpu_count() or 1))
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -389,7 +389,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--heads", type=int, default=0, help="profiling only: run a subset of the workload's heads")
     args = ap.parse_args()
-    cfg = inputs.CONFIGS[args.workload]
+    cfg = {**inputs.CONFIGS, **inputs.PAPER_SCALE_CONFIGS}[args.workload]
     if args.heads > 0:
         cfg = cfg.replace(H=args.heads, name=f"{cfg.name}[{args.heads} heads]")
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -369,8 +369,25 @@ void launch_kmeans_norms(const KmArgs &a, cudaStream_t st)
 void launch_kmeans_iteration(const KmArgs &a, int32_t *status, cudaStream_t st)
 {
     const char *force = getenv("SCOPE_KMEANS_SIMT");  // testing aid: run the general kernel
-    if (kmeans_tc_supported(a, nullptr) && !(force && force[0] == '1')) {
+    const bool simt = force && force[0] == '1';
+    // the three key ranges in one launch if their codebooks fit shared and tensor memory together, else one
+    // launch per range (codebooks of a few hundred centroids), else the general kernel
+    bool per_range = !simt && a.nspaces == 3 && a.codes != nullptr;
+    KmArgs one[3];
+    for (int m = 0; m < 3 && per_range; ++m) {
+        one[m] = a;
+        one[m].nspaces = 1;
+        one[m].sp[0] = a.sp[m];
+        one[m].single_field = m + 1;
+        one[m].assign = nullptr;
+        one[m].x2_ready = a.x2_ready || m > 0;  // the first launch of a call leaves the row norms for the rest
+        per_range = kmeans_tc_supported(one[m], nullptr);
+    }
+    if (!simt && kmeans_tc_supported(a, nullptr)) {
         launch_kmeans_assign_tc(a, status, st);
+    } else if (per_range) {
+        for (int m = 0; m < 3; ++m)
+            launch_kmeans_assign_tc(one[m], status, st);
     } else {
         dim3 grid((a.N + TM - 1) / TM, a.B * a.H);
         kmeans_assign_kernel<<<grid, NT, 0, st>>>(a);

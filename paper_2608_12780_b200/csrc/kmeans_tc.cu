@@ -28,11 +28,14 @@ constexpr int NT = 128 * MAX_GROUPS;
 constexpr int HALF_BYTES = TM * 128;           // one 64-channel half of a 128-row tile
 constexpr int XTILE_BYTES = 2 * HALF_BYTES;    // 32 KB
 
+constexpr int MAXC = 512;      // centroids per range this kernel holds (two MMAs of up to 256 columns)
+constexpr int MAXC_ALL = 768;  // ... and over all ranges of one launch
+
 struct TcLayout {
     int cpad[3];       // centroids padded to a multiple of 16
-    int col[3];        // first TMEM column of the space inside a group's 256
+    int col[3];        // first TMEM column of the space inside a pipeline's columns
     int cent_off[3];   // byte offset of the space's split tiles in shared memory
-    int un_off[3];     // float offset of the space's norms
+    int un_off[3];     // float offset of the space's norms = first label slot of the range in the per-tile tables
     int cent_bytes;    // all split tiles
     int un_floats;
     int cols;          // TMEM columns one pipeline needs (multiple of 32)
@@ -43,7 +46,7 @@ __host__ __device__ inline bool tc_layout(const KmArgs &a, TcLayout &L)
     int col = 0, off = 0, un = 0;
     for (int s = 0; s < a.nspaces; ++s) {
         int cp = (a.sp[s].C + 15) & ~15;
-        if (cp > 256)
+        if (cp > MAXC)
             return false;
         L.cpad[s] = cp;
         L.col[s] = col;
@@ -56,22 +59,21 @@ __host__ __device__ inline bool tc_layout(const KmArgs &a, TcLayout &L)
     L.cent_bytes = off;
     L.un_floats = un;
     L.cols = col;
-    return col <= 256;
+    return col <= 512 && un <= MAXC_ALL;
 }
 
-constexpr int MAXC = 256;  // centroids per range this kernel holds
 constexpr int MAXCAND = 128;  // (token, contender) pairs re-evaluated by one thread each, per tile
 
 struct GroupShared {
     uint16_t asg[3][TM];         // label of every token of the tile, per range
-    uint32_t cnt[3][MAXC / 4];   // members per label in this tile, four 8-bit counters per word (a tile has 128 tokens)
-    uint8_t start[3][MAXC];      // first slot of the label's run
+    uint32_t cnt[MAXC_ALL / 4];  // members per label in this tile (ranges back to back), four 8-bit counters per word
+    uint8_t start[MAXC_ALL];     // first slot of the label's run
     uint32_t runs[3][TM];        // non-empty labels: label | start << 10 | count << 18
     int nruns[3];
     uint16_t sorted[3][TM];      // tokens of the tile grouped by label, as the row part of their shared-memory address
     uint16_t flagged[3 * TM];    // range << 8 | token: close calls that are re-evaluated against every centroid
     int nflagged;
-    uint32_t cand[MAXCAND];      // close calls with at most four contenders: centroid | token << 8 | range << 15 | k << 17 | n << 19
+    uint32_t cand[MAXCAND];      // close calls with at most four contenders: centroid | token << 10 | range << 17 | k << 19 | n << 21
     double cdist[MAXCAND];       // fp64 distance of each contender
     int ncand;
     int next_tile;               // the tile this pipeline takes after the current one
@@ -179,22 +181,25 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             G.ncand = 0;
             for (int s = 0; s < a.nspaces; ++s) {
                 const int cp = L.cpad[s];
-                const uint32_t idesc = idesc_bf16(TM, cp, false, false);
                 const int k_lo = a.sp[s].ch0 >> 4, k_hi = (a.sp[s].ch0 + a.sp[s].D + 15) >> 4;
                 const uint32_t cb = smem_u32(s_cent) + L.cent_off[s];
-                bool acc = false;
-                for (int p = 0; p < NSPLIT; ++p)
-                    for (int ks = k_lo; ks < k_hi; ++ks) {
-                        const uint32_t ao = (xbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4;
-                        const uint32_t bo = (cb + (p * 2 + (ks >> 2)) * cp * 128 + (ks & 3) * 32) >> 4;
-                        mma_ss2(tmem_g + L.col[s], d_lo + ao, d_hi, d_lo + bo, d_hi, idesc, acc);
-                        acc = true;
-                    }
+                // one instruction covers up to 256 centroids: larger codebooks take two column blocks
+                for (int n0 = 0; n0 < cp; n0 += 256) {
+                    const uint32_t idesc = idesc_bf16(TM, min(256, cp - n0), false, false);
+                    bool acc = false;
+                    for (int p = 0; p < NSPLIT; ++p)
+                        for (int ks = k_lo; ks < k_hi; ++ks) {
+                            const uint32_t ao = (xbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4;
+                            const uint32_t bo = (cb + ((p * 2 + (ks >> 2)) * cp + n0) * 128 + (ks & 3) * 32) >> 4;
+                            mma_ss2(tmem_g + L.col[s] + n0, d_lo + ao, d_hi, d_lo + bo, d_hi, idesc, acc);
+                            acc = true;
+                        }
+                }
             }
             mma_commit(&G.mbar);
         }
-        for (int e = gt; e < a.nspaces * (MAXC / 4); e += 128)
-            (&G.cnt[0][0])[e] = 0u;
+        for (int e = gt; e < MAXC_ALL / 4; e += 128)
+            G.cnt[e] = 0u;
         // squared norm of the whole row (an upper bound of every range's slice, used in the tolerance): taken
         // from the tile in the first pass of a call and kept in global memory for the later ones
         float x2 = 0.f;
@@ -289,7 +294,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                     // warp-wide, so the whole warp walks it).  Usually two.
                     const float lim = best + tol;
                     int nc = 0;
-                    uint32_t packed = 0;
+                    unsigned long long packed = 0;
                     for (int c0 = 0; c0 < cp; c0 += 32) {
                         uint32_t r[32];
                         if (cp - c0 >= 32) {
@@ -311,7 +316,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                                 const float dist = fmaf(-2.f, __uint_as_float(r[j]), un[c0 + j]);
                                 if (close && dist <= lim) {
                                     if (nc < 4)
-                                        packed |= (uint32_t)(c0 + j) << (8 * nc);
+                                        packed |= (unsigned long long)(c0 + j) << (16 * nc);
                                     ++nc;
                                 }
                             }
@@ -323,11 +328,11 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                             base = atomicAdd(&G.ncand, nc);
                         if (base + nc <= MAXCAND) {
                             for (int k = 0; k < nc; ++k)
-                                G.cand[base + k] = ((packed >> (8 * k)) & 0xffu) | ((uint32_t)gt << 8) | ((uint32_t)s << 15) |
-                                                   ((uint32_t)k << 17) | ((uint32_t)nc << 19);
+                                G.cand[base + k] = (uint32_t)((packed >> (16 * k)) & 0x3ffu) | ((uint32_t)gt << 10) | ((uint32_t)s << 17) |
+                                                   ((uint32_t)k << 19) | ((uint32_t)nc << 21);
                         } else {  // many contenders (or a full list): every centroid is re-evaluated
                             for (int k = base; k < MAXCAND; ++k)
-                                G.cand[k] = 1u << 17;  // reserved but unused slots: never the first of a token
+                                G.cand[k] = 1u << 19;  // reserved but unused slots: never the first of a token
                             int slot = atomicAdd(&G.nflagged, 1);
                             G.flagged[slot] = (uint16_t)((s << 8) | gt);
                         }
@@ -350,7 +355,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             if (ncand > 0) {
                 if (gt < ncand) {
                     const uint32_t e = G.cand[gt];
-                    const int c = e & 0xff, lt = (e >> 8) & 0x7f, s = (e >> 15) & 3;
+                    const int c = e & 0x3ff, lt = (e >> 10) & 0x7f, s = (e >> 17) & 3;
                     const KmSpace &sp = a.sp[s];
                     const float *u = sp.cent + ((size_t)bh * sp.C + c) * sp.D;
                     double d = 0.0;
@@ -367,14 +372,14 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                 bar_sync(1 + grp, 128);
                 if (gt < ncand) {
                     const uint32_t e = G.cand[gt];
-                    if (((e >> 17) & 3) == 0) {  // first contender of its token: ascending centroid order, lowest wins ties
-                        const int n = (e >> 19) & 7, lt = (e >> 8) & 0x7f, s = (e >> 15) & 3;
+                    if (((e >> 19) & 3) == 0) {  // first contender of its token: ascending centroid order, lowest wins ties
+                        const int n = (e >> 21) & 7, lt = (e >> 10) & 0x7f, s = (e >> 17) & 3;
                         double bd = G.cdist[gt];
-                        int ba = e & 0xff;
+                        int ba = e & 0x3ff;
                         for (int k = 1; k < n; ++k)
                             if (G.cdist[gt + k] < bd) {
                                 bd = G.cdist[gt + k];
-                                ba = G.cand[gt + k] & 0xff;
+                                ba = G.cand[gt + k] & 0x3ff;
                             }
                         G.asg[s][lt] = (uint16_t)ba;
                     }
@@ -429,13 +434,19 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             for (int s = 0; s < a.nspaces; ++s) {
                 lab[s] = G.asg[s][gt];
                 const int sh = (lab[s] & 3) * 8;
-                pos[s] = (int)((atomicAdd(&G.cnt[s][lab[s] >> 2], 1u << sh) >> sh) & 0xffu);
+                pos[s] = (int)((atomicAdd(&G.cnt[(L.un_off[s] + lab[s]) >> 2], 1u << sh) >> sh) & 0xffu);
             }
-            if (a.nspaces == 1)
-                a.assign[(size_t)bh * a.N + tok0 + gt] = lab[0];
-            else
-                a.codes[(size_t)bh * a.N + tok0 + gt] =
-                    (uint32_t)lab[0] | ((uint32_t)lab[1] << kCodeBits) | ((uint32_t)lab[2] << (2 * kCodeBits));
+            const size_t at = (size_t)bh * a.N + tok0 + gt;
+            if (a.single_field > 0) {
+                // one range of the keys per launch (T, then H, then W): the first rewrites the word, the others their field
+                const int sh = (a.single_field - 1) * kCodeBits;
+                a.codes[at] = a.single_field == 1 ? (uint32_t)lab[0]
+                                                  : ((a.codes[at] & ~((uint32_t)kCodeMask << sh)) | ((uint32_t)lab[0] << sh));
+            } else if (a.nspaces == 1) {
+                a.assign[at] = lab[0];
+            } else {
+                a.codes[at] = (uint32_t)lab[0] | ((uint32_t)lab[1] << kCodeBits) | ((uint32_t)lab[2] << (2 * kCodeBits));
+            }
         }
         bar_sync(1 + grp, 128);
         if (gw < a.nspaces) {
@@ -444,7 +455,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             int base = 0, nr = 0;
             for (int c0 = 0; c0 < cp; c0 += 32) {
                 const int c = c0 + lane;
-                const int n = c < cp ? (int)((G.cnt[s][c >> 2] >> ((c & 3) * 8)) & 0xffu) : 0;
+                const int n = c < cp ? (int)((G.cnt[(L.un_off[s] + c) >> 2] >> ((c & 3) * 8)) & 0xffu) : 0;
                 int inc = n;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -454,7 +465,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                 }
                 const int st = base + inc - n;
                 if (c < cp)
-                    G.start[s][c] = (uint8_t)st;
+                    G.start[L.un_off[s] + c] = (uint8_t)st;
                 const uint32_t m = __ballot_sync(0xffffffffu, n > 0);
                 if (n > 0)
                     G.runs[s][nr + __popc(m & ((1u << lane) - 1u))] = (uint32_t)c | ((uint32_t)st << 10) | ((uint32_t)n << 18);
@@ -467,7 +478,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         bar_sync(1 + grp, 128);
         if (valid)
             for (int s = 0; s < a.nspaces; ++s)
-                G.sorted[s][G.start[s][lab[s]] + pos[s]] = (uint16_t)sw128(gt, 0);
+                G.sorted[s][G.start[L.un_off[s] + lab[s]] + pos[s]] = (uint16_t)sw128(gt, 0);
         bar_sync(1 + grp, 128);
 
         // ---- member sums: a thread owns two adjacent channels (one 32-bit word of every row) and every other
@@ -484,7 +495,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             // sw128(row, chunk) = sw128(row, 0) ^ (chunk << 4): the sorted list holds the row part
             const uint32_t xpair = xbase + (ch >> 6) * HALF_BYTES + (ch & 7) * 2;
             const uint32_t cbits = (uint32_t)((ch & 63) >> 3) << 4;
-            const int nr = G.nruns[s];
+            const int nr = (rel >= 0 && rel < sp.D) ? G.nruns[s] : 0;  // a one-range launch leaves the other channels alone
             for (int r = hf; r < nr; r += 2) {
                 const uint32_t run = G.runs[s][r];
                 const int cl = run & 1023, st = (run >> 10) & 255, n = run >> 18;

@@ -43,6 +43,7 @@ struct KmArgs {
     uint32_t *codes;   // [BH, N] packed labels (nspaces == 3)
     float *x2;         // [BH, N] squared row norms, kept from the first pass to the later ones (may be null)
     int x2_ready;      // 0: this pass computes and stores them, 1: it reads them
+    int single_field;  // 0: outputs as nspaces says; m + 1: a one-range launch that writes field m of the packed codes
 };
 
 // Per (head, query cluster) result of the selection stage that later kernels read.

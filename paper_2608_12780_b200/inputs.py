@@ -71,6 +71,14 @@ CONFIGS = {
     "HY720": ScopeConfig("HY720", 1, 24, (33, 45, 80), (16, 56, 56), 128, 16, 64, 64, 5, 0.9, 512),
 }
 
+# The same two 720p shapes with the hyper-parameters the paper's experiments state (Section 5.1: 300 query
+# clusters, 333 centroids per key subspace, floor = ceil(0.1 N)): non-power-of-two codebooks, codes above 8 bits,
+# tables that no longer fit shared memory whole.
+PAPER_SCALE_CONFIGS = {
+    "W720P": ScopeConfig("W720P", 1, 40, (21, 45, 80), (44, 42, 42), 300, 333, 333, 333, 5, 0.9, 7560),
+    "HY720P": ScopeConfig("HY720P", 1, 24, (33, 45, 80), (16, 56, 56), 300, 333, 333, 333, 5, 0.9, 11880),
+}
+
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """Round-to-nearest-even fp32 -> bf16, returned as uint16 bit patterns."""

@@ -315,12 +315,17 @@ def test_kmeans_general_kernel_path(monkeypatch):
     _compare_plan(plan2, ref, cfg)
 
 
-def test_large_codebooks_use_general_kernel():
-    """More centroids than the tensor-core kernel holds (C > 256): still exact."""
-    cfg = inputs.ScopeConfig("bigC", 1, 1, (6, 10, 10), (16, 56, 56), 300, 8, 272, 16, 2, 0.9, 32)
+@pytest.mark.parametrize("Cq,Ct,Ch,Cw", [
+    (300, 8, 272, 16),     # tensor-core kernel, codebooks above 256 take two column blocks per MMA step
+    (300, 333, 333, 333),  # the paper's codebook sizes: the three key ranges run as one launch each
+    (32, 8, 520, 16),      # more centroids than the tensor-core kernel holds: general kernel
+])
+def test_large_codebooks(Cq, Ct, Ch, Cw):
+    """Codebooks of a few hundred centroids (non-power-of-two, codes above 8 bits): still exact."""
+    cfg = inputs.ScopeConfig("bigC", 1, 2, (6, 10, 10), (16, 56, 56), Cq, Ct, Ch, Cw, 3, 0.9, 32)
     Q, K, V, dQ, dK, dV = _layer(cfg, 8)
     ref = _oracle_plans(Q, K, cfg)
-    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.Cq * cfg.N))
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.H * cfg.Cq * cfg.N))
     sb.scope_plan(dQ, dK, plan)
     plan.check()
     _compare_plan(plan, ref, cfg)
