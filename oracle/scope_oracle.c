@@ -18,6 +18,8 @@
  *   scope_oracle_key_set     the set S_c of Eq. 10
  *   scope_oracle_attn_row    one output row of Eq. 11
  *   scope_oracle_dense_row   one output row of Eq. 1
+ *   scope_oracle_recall_row  how much of a query's exact attention a key set keeps (the quantity of the
+ *                            recall figure and of the matched-oracle-recall protocol in the supplement)
  *
  * Readings taken where the paper is silent (also listed in the design notes):
  * evenly strided initial centroids, a fixed number of Lloyd iterations, squared
@@ -343,5 +345,65 @@ int scope_oracle_dense_row(const uint16_t *q, const uint16_t *K, const uint16_t 
         out[ch] = (float)(acc[ch] / Z);
     free(logit);
     free(acc);
+    return 0;
+}
+
+/* Recall diagnostics for one query.  With a_j the weights of Eq. 1 over all N keys:
+ *   mass        = sum of a_j over j in S (attention recall of the set S);
+ *   n_important = number of keys whose exact logit is at least the T-th largest, T = ceil(top_frac N)
+ *                 (keys tied with the T-th are all counted);
+ *   top_recall  = share of those keys that S contains.
+ * Logits are the plain sequential fp64 dot product times the scale; S holds distinct key indices. */
+static int dbl_desc_cmp(const void *a, const void *b)
+{
+    const double x = *(const double *)a, y = *(const double *)b;
+    return x > y ? -1 : (x < y ? 1 : 0);
+}
+
+int scope_oracle_recall_row(const uint16_t *q, const uint16_t *K, int64_t row_stride, int d, int64_t N,
+                            const int32_t *S, int64_t len, float scale, double top_frac,
+                            double *mass, double *top_recall, int64_t *n_important)
+{
+    double *logit = (double *)malloc(sizeof(double) * (size_t)N);
+    double *sorted = (double *)malloc(sizeof(double) * (size_t)N);
+    if (!logit || !sorted) {
+        free(logit);
+        free(sorted);
+        return -1;
+    }
+    double mx = -INFINITY;
+    for (int64_t j = 0; j < N; ++j) {
+        double dot = 0.0;
+        for (int ch = 0; ch < d; ++ch)
+            dot += (double)bf16_to_f32(q[ch]) * (double)bf16_to_f32(K[j * row_stride + ch]);
+        logit[j] = dot * (double)scale;
+        if (logit[j] > mx)
+            mx = logit[j];
+    }
+    double Z = 0.0;
+    for (int64_t j = 0; j < N; ++j)
+        Z += exp(logit[j] - mx);
+    double kept = 0.0;
+    for (int64_t l = 0; l < len; ++l)
+        kept += exp(logit[S[l]] - mx);
+    *mass = kept / Z;
+
+    int64_t T = (int64_t)ceil(top_frac * (double)N);
+    if (T < 1)
+        T = 1;
+    if (T > N)
+        T = N;
+    memcpy(sorted, logit, sizeof(double) * (size_t)N);
+    qsort(sorted, (size_t)N, sizeof(double), dbl_desc_cmp);
+    const double thr = sorted[T - 1];
+    int64_t important = 0, hit = 0;
+    for (int64_t j = 0; j < N; ++j)
+        important += logit[j] >= thr;
+    for (int64_t l = 0; l < len; ++l)
+        hit += logit[S[l]] >= thr;
+    *n_important = important;
+    *top_recall = (double)hit / (double)important;
+    free(logit);
+    free(sorted);
     return 0;
 }

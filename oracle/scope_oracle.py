@@ -41,6 +41,8 @@ def lib():
         L.scope_oracle_attn_row.restype = C.c_int
         L.scope_oracle_dense_row.argtypes = [p, p, p, C.c_int64, C.c_int, C.c_int64, C.c_float, p]
         L.scope_oracle_dense_row.restype = C.c_int
+        L.scope_oracle_recall_row.argtypes = [p, p, C.c_int64, C.c_int, C.c_int64, p, C.c_int64, C.c_float, C.c_double, p, p, p]
+        L.scope_oracle_recall_row.restype = C.c_int
         _lib = L
     return _lib
 
@@ -229,6 +231,27 @@ def dense_rows(Q, K, V, scale: float, rows) -> np.ndarray:
             raise MemoryError
         out[n] = o
     return out
+
+
+def recall_rows(Q, K, g, S, scale: float, rows, top_frac: float):
+    """Recall diagnostics of the key set of each listed query (its cluster's S_c) against the exact logits of
+    Eq. 1: (attention mass kept, share of the keys at or above the ceil(top_frac N)-th largest logit kept,
+    number of such keys)."""
+    Q, K = _u16(Q), _u16(K)
+    N, d = Q.shape
+    rows = np.asarray(rows, np.int64)
+    mass = np.empty(rows.shape[0], np.float64)
+    top = np.empty(rows.shape[0], np.float64)
+    nimp = np.empty(rows.shape[0], np.int64)
+    m, t, n = C.c_double(), C.c_double(), C.c_int64()
+    for k, i in enumerate(rows):
+        Sc = np.ascontiguousarray(S[int(g[i])], np.int32)
+        rc = lib().scope_oracle_recall_row(_ptr(Q[i]), _ptr(K), d, d, N, _ptr(Sc), Sc.shape[0], np.float32(scale),
+                                           float(top_frac), C.byref(m), C.byref(t), C.byref(n))
+        if rc != 0:
+            raise MemoryError
+        mass[k], top[k], nimp[k] = m.value, t.value, n.value
+    return mass, top, nimp
 
 
 def forward_head(Q, K, V, p):

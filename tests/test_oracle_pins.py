@@ -399,3 +399,46 @@ def test_selection_variants_of_the_ablation():
     for c in range(cfg.Cq):  # nested along one ranking: pure Top-p <= fixed hybrid <= online
         assert set(Sp[c].tolist()) <= set(Sf[c].tolist()) <= set(S[c].tolist())
     assert (r > b).any()  # the online rule extends some cluster in this case
+
+
+# ----------------------------------------------------------------------------- recall diagnostics
+
+
+def test_recall_toy_matches_hand_worked():
+    """Four keys with logits 2, 1, 1, 0 (query e_1, unit scale): weights e^2, e, e, 1.  S = {0, 3} keeps
+    (e^2 + 1) / (e^2 + 2e + 1) of the mass; with top_frac = 1/2 the second-largest logit is 1, so keys 0, 1, 2
+    are the important ones (the tie counts) and S holds one of the three."""
+    Q = _bits(np.array([[1.0, 0.0]] * 4))
+    K = _bits(np.array([[2.0, 5.0], [1.0, -3.0], [1.0, 7.0], [0.0, 1.0]]))
+    g = np.zeros(4, np.int32)
+    S = [np.array([0, 3], np.int32)]
+    mass, top, nimp = orc.recall_rows(Q, K, g, S, 1.0, [0], 0.5)
+    e = math.e
+    assert abs(mass[0] - (e * e + 1) / (e * e + 2 * e + 1)) < 1e-15
+    assert nimp[0] == 3 and top[0] == 1.0 / 3.0
+    # the whole key set keeps everything
+    mass, top, nimp = orc.recall_rows(Q, K, g, [np.arange(4, dtype=np.int32)], 1.0, [1], 0.25)
+    assert mass[0] == 1.0 and top[0] == 1.0 and nimp[0] == 1
+
+
+def test_recall_against_sorted_softmax():
+    cfg, Q, K, V = _head("tiny", seed=6)
+    pl = orc.plan_head(Q, K, cfg)
+    rows = np.arange(0, cfg.N, 17)
+    frac = 0.1
+    mass, top, nimp = orc.recall_rows(Q, K, pl.g, pl.S, cfg.scale, rows, frac)
+    logits = (_f32(Q).astype(np.float64) @ _f32(K).astype(np.float64).T) * float(np.float32(cfg.scale))
+    T = math.ceil(frac * cfg.N)
+    for k, i in enumerate(rows):
+        a = np.exp(logits[i] - logits[i].max())
+        a /= a.sum()
+        Sc = pl.S[pl.g[i]]
+        assert abs(mass[k] - a[Sc].sum()) < 1e-12
+        order = np.argsort(-logits[i], kind="stable")
+        assert nimp[k] == T  # no ties among random logits
+        assert top[k] == np.isin(order[:T], Sc).sum() / T
+    assert np.all(mass > 0.0) and np.all(mass <= 1.0 + 1e-15)
+    # rho = 1 selects every key
+    full = orc.plan_head(Q, K, cfg.replace(top_p=1.0))
+    mass, top, _ = orc.recall_rows(Q, K, full.g, full.S, cfg.scale, rows, frac)
+    assert np.all(np.abs(mass - 1.0) < 1e-15) and np.all(top == 1.0)
