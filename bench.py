@@ -273,6 +273,23 @@ def run_scope(args, cfg):
     stage_ms["group"] = time_stage(lambda: sb.scope_plan_stages(None, None, plan, sb.STAGE_GROUP))
     stage_ms["sparse_attn"] = time_stage(lambda: sb.scope_sparse_attn(dQ, dK, dV, plan, dO))
 
+    # ---- recall diagnostics of the plan just timed (outside the timed region): a few queries per head against
+    # the exact logits of Eq. 1
+    recall = None
+    if args.recall_rows > 0 and rank == 0:
+        sb.scope_plan(dQ, dK, plan)
+        rng = np.random.default_rng(args.seed + 1)
+        rr = np.stack([np.sort(rng.choice(cfg.N, args.recall_rows, replace=False)) for _ in range(cfg.H)])
+        rows_t = torch.from_numpy(rr[None].astype(np.int32)).to(dev)
+        mass, top = sb.scope_recall(dQ, dK, plan, rows_t, 0.1)
+        plan.check("recall diagnostics")
+        mass, top = mass.cpu().numpy().ravel(), top.cpu().numpy().ravel()
+        recall = {"rows_per_head": args.recall_rows, "attention_mass_mean": float(mass.mean()),
+                  "attention_mass_median": float(np.median(mass)), "attention_mass_min": float(mass.min()),
+                  "top10pct_keys_kept_mean": float(top.mean()), "retention": density,
+                  "note": "exact fp64 logits of sampled queries vs the key set of their cluster; synthetic inputs"}
+        del mass, top, rows_t
+
     # ---- dense comparator: Eq. 1 through the same kernel on a few heads, scaled to the layer
     dense_ms = None
     if args.dense_heads > 0 and rank == 0:
@@ -359,6 +376,7 @@ def run_scope(args, cfg):
             "select_gbs": sel_bytes / (stage_ms["select"] * 1e-3) / 1e9,
             "kmeans_gbs": cfg.iters * 2 * nbytes / ((stage_ms["kmeans_q"] + stage_ms["kmeans_k"]) * 1e-3) / 1e9,
             "dense_attn_ms_same_kernel": dense_ms,
+            "recall": recall,
             "plan_stats": {"density": density, "selected_pairs": pairs, "index_entries": int(need),
                            "k_head_min_med_max": [int(k_head.min()), int(np.median(k_head)), int(k_head.max())],
                            "t_c_min_med_max": [int(t_c.min()), int(np.median(t_c)), int(t_c.max())],
@@ -387,6 +405,7 @@ def main():
     ap.add_argument("--e2e-groups", type=int, default=4, help="head groups (plans / streams) of the host path")
     ap.add_argument("--dense-heads", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--recall-rows", type=int, default=8, help="sampled queries per head for the recall diagnostics (0: skip)")
     ap.add_argument("--heads", type=int, default=0, help="profiling only: run a subset of the workload's heads")
     args = ap.parse_args()
     cfg = {**inputs.CONFIGS, **inputs.PAPER_SCALE_CONFIGS}[args.workload]

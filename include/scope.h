@@ -171,6 +171,24 @@ scope_status scope_forward_host_async(const void *Q_host, const void *K_host, co
 scope_status scope_dense_attn(const void *Q, const void *K, const void *V, const scope_plan_t *plan,
                               void *O, void *stream);
 
+/* Recall diagnostics of a finished plan (the quantity of the paper's recall figure, and the
+ * retention-versus-oracle-recall protocol of its supplement, Section "Fine-Grained Key Selection at
+ * Matched Oracle Recall").  For each sampled query i (cluster c = g_i) and the exact attention
+ * weights a_ij of Eq. 1 over all N keys:
+ *   mass[i]       = sum of a_ij over j in S_c                     (attention recall);
+ *   top_recall[i] = |S_c ∩ I_i| / |I_i|, I_i = the keys whose exact logit is at least the T-th
+ *                   largest of the row, T = ceil(top_frac * N), ties with the T-th included.
+ * Retention is r_c / N (SCOPE_FIELD_FINAL_COUNT).
+ * rows: DEVICE int32 [B*H, rows_per_head] token indices in [0, N); an index outside the range gives
+ * NaN outputs for that row and SCOPE_ERR_INVALID_ARG in the status word.  scratch: DEVICE memory of
+ * scope_recall_scratch_bytes() bytes, owned by the caller, 16-byte aligned.  mass, top_recall:
+ * DEVICE double [B*H * rows_per_head].  Logits are fp64 (sequential dot product over the channels).
+ * Asynchronous on `stream`; not part of the timed layer. */
+size_t scope_recall_scratch_bytes(const scope_params *params, int32_t rows_per_head);
+scope_status scope_recall(const void *Q, const void *K, const scope_plan_t *plan, const int32_t *rows,
+                          int32_t rows_per_head, double top_frac, void *scratch, size_t scratch_bytes,
+                          double *mass, double *top_recall, void *stream);
+
 /* Synchronise `stream` and read the device status word.  Returns SCOPE_OK,
  * SCOPE_ERR_CAPACITY (then *needed_capacity, if not NULL, receives the number of
  * index entries the last plan needs), SCOPE_ERR_BAD_PLAN, SCOPE_ERR_TIMEOUT or

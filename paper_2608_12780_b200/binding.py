@@ -31,7 +31,7 @@ EXPORTS = ["scope_plan_workspace_bytes", "scope_plan_create", "scope_plan_destro
            "scope_sparse_attn", "scope_forward", "scope_forward_host", "scope_forward_host_async", "scope_dense_attn", "scope_plan_status",
            "scope_plan_reset_status", "scope_plan_get", "scope_plan_field_bytes", "scope_plan_export",
            "scope_plan_import", "scope_status_string", "scope_kfix_from_alpha", "scope_kernel_launches",
-           "scope_kmeans_queries_static"]
+           "scope_kmeans_queries_static", "scope_recall_scratch_bytes", "scope_recall"]
 
 
 class ScopeParams(C.Structure):
@@ -72,6 +72,9 @@ def lib():
         L.scope_sparse_attn.argtypes = [vp, vp, vp, vp, vp, vp]
         L.scope_dense_attn.argtypes = [vp, vp, vp, vp, vp, vp]
         L.scope_forward.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.scope_recall_scratch_bytes.argtypes = [vp, C.c_int32]
+        L.scope_recall_scratch_bytes.restype = sz
+        L.scope_recall.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_double, vp, sz, vp, vp, vp]
         L.scope_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
         L.scope_forward_host_async.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
         L.scope_plan_status.argtypes = [vp, vp, C.POINTER(i64)]
@@ -248,6 +251,25 @@ def scope_dense_attn(Q, K, V, plan: Plan, O=None):
     _check(lib().scope_dense_attn(_dev_ptr(Q, "Q"), _dev_ptr(K, "K"), _dev_ptr(V, "V"), plan.handle,
                                   _dev_ptr(O, "O"), C.c_void_p(_stream())), "scope_dense_attn")
     return O
+
+
+def scope_recall(Q, K, plan: Plan, rows: torch.Tensor, top_frac: float = 0.1):
+    """Recall diagnostics of a finished plan for the sampled queries ``rows`` (int32 [B, H, R] token indices on
+    the device): (attention mass kept, share of the keys at or above the ceil(top_frac N)-th largest exact logit
+    kept), both float64 [B, H, R]."""
+    p = plan.params
+    if rows.dtype != torch.int32 or not rows.is_cuda or not rows.is_contiguous() or rows.dim() != 3 \
+            or rows.shape[0] != p.B or rows.shape[1] != p.H:
+        raise ValueError("rows: contiguous int32 CUDA tensor [B, H, R]")
+    R = int(rows.shape[2])
+    nbytes = lib().scope_recall_scratch_bytes(C.byref(p), R)
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=rows.device)
+    mass = torch.empty(rows.shape, dtype=torch.float64, device=rows.device)
+    top = torch.empty(rows.shape, dtype=torch.float64, device=rows.device)
+    _check(lib().scope_recall(_dev_ptr(Q, "Q"), _dev_ptr(K, "K"), plan.handle, C.c_void_p(rows.data_ptr()), R,
+                              float(top_frac), C.c_void_p(scratch.data_ptr()), nbytes, C.c_void_p(mass.data_ptr()),
+                              C.c_void_p(top.data_ptr()), C.c_void_p(_stream())), "scope_recall")
+    return mass, top
 
 
 def scope_forward(Q, K, V, plan: Plan, O=None):

@@ -422,6 +422,48 @@ scope_status scope_sparse_attn(const void *Q, const void *K, const void *V, cons
     return attn_common(Q, K, V, plan, O, stream, 0);
 }
 
+size_t scope_recall_scratch_bytes(const scope_params *params, int32_t rows_per_head)
+{
+    if (!params || rows_per_head <= 0 || params->B <= 0 || params->H <= 0 || params->N <= 0)
+        return 0;
+    return (size_t)params->B * params->H * (size_t)rows_per_head * (size_t)params->N * sizeof(double);
+}
+
+scope_status scope_recall(const void *Q, const void *K, const scope_plan_t *pl, const int32_t *rows,
+                          int32_t rows_per_head, double top_frac, void *scratch, size_t scratch_bytes,
+                          double *mass, double *top_recall, void *stream)
+{
+    if (!pl || !Q || !K || !rows || !scratch || !mass || !top_recall || rows_per_head <= 0)
+        return SCOPE_ERR_INVALID_ARG;
+    if (!(top_frac > 0.0) || !(top_frac <= 1.0))
+        return SCOPE_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(scratch))
+        return SCOPE_ERR_ALIGNMENT;
+    const scope_params &p = pl->p;
+    if (scratch_bytes < scope_recall_scratch_bytes(&p, rows_per_head))
+        return SCOPE_ERR_WORKSPACE;
+    RecallArgs a{};
+    a.Q = static_cast<const bf16 *>(Q);
+    a.K = static_cast<const bf16 *>(K);
+    a.sb = p.stride_b; a.sh = p.stride_h; a.sn = p.stride_n;
+    a.B = p.B; a.H = p.H; a.N = p.N; a.Cq = p.Cq;
+    a.scale = p.scale;
+    a.rows = rows;
+    a.rows_per_head = rows_per_head;
+    long long T = (long long)ceil(top_frac * (double)p.N);
+    a.top_count = T < 1 ? 1 : (T > p.N ? p.N : T);
+    a.logits = static_cast<double *>(scratch);
+    a.g = pl->q_assign;
+    a.r_c = pl->r_c;
+    a.key_offsets = pl->key_offsets;
+    a.key_indices = pl->key_indices;
+    a.mass = mass;
+    a.top_recall = top_recall;
+    a.status = pl->status;
+    launch_recall(a, static_cast<cudaStream_t>(stream));
+    return cuda_ok(cudaGetLastError());
+}
+
 scope_status scope_dense_attn(const void *Q, const void *K, const void *V, const scope_plan_t *plan, void *O,
                               void *stream)
 {

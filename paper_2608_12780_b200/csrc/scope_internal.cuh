@@ -111,6 +111,25 @@ void launch_select(const SelectArgs &a, cudaStream_t st);
 void launch_group(const GroupArgs &a, cudaStream_t st);
 void launch_tiles_from_offsets(const GroupArgs &a, cudaStream_t st);
 void launch_attn(const AttnArgs &a, cudaStream_t st);
+
+// Recall diagnostics (recall.cu): sampled queries against the exact logits of Eq. 1.
+struct RecallArgs {
+    const bf16 *Q, *K;
+    int64_t sb, sh, sn;
+    int B, H, N, Cq;
+    float scale;
+    const int32_t *rows;       // [BH, rows_per_head] token indices (device)
+    int rows_per_head;
+    long long top_count;       // T: the important keys are those at or above the T-th largest logit
+    double *logits;            // [BH * rows_per_head, N] scratch
+    const int32_t *g;          // [BH, N] query labels
+    const int32_t *r_c;        // [BH, Cq]
+    const int64_t *key_offsets;
+    const int32_t *key_indices;
+    double *mass, *top_recall; // [BH * rows_per_head]
+    int32_t *status;
+};
+void launch_recall(const RecallArgs &a, cudaStream_t st);
 constexpr int kAttnTileRows = 256;
 
 void count_launch(int n = 1);

@@ -4,7 +4,8 @@ heads and rows the CPU oracle can compute one by one.
 Per sampled head: the end-to-end plan of the CUDA path against the oracle's (labels, counts,
 per-head k, key sets), the selection stage fed the oracle's codes / tables / cluster sizes
 (selected-mask Jaccard >= 0.999 per cluster, the bar for large shapes), and the attention output of
-sampled query rows given the CUDA path's own key sets (max-abs 2e-2, relative L2 1e-2).
+sampled query rows given the CUDA path's own key sets (max-abs 2e-2, relative L2 1e-2), and the
+recall diagnostics of sampled queries (top-key share identical, attention mass to 1e-11).
 """
 import numpy as np
 import pytest
@@ -60,6 +61,13 @@ def test_full_size_layer_on_sampled_heads(name, heads):
     assert np.array_equal(sub.export("K_HEAD"), np.array([p.k_head for p in ref]))
     assert np.array_equal(sub.export("TOPP_COUNT"), st(lambda p: p.t_c))
 
+    # recall diagnostics of sampled queries of every head (checked below on the sampled heads)
+    rrng = np.random.default_rng(2)
+    rrows = np.stack([np.sort(rrng.choice(N, 6, replace=False)) for _ in range(cfg.H)]).astype(np.int32)
+    mass, top = sb.scope_recall(dQ, dK, plan, torch.from_numpy(rrows[None]).cuda(), 0.1)
+    plan.check()
+    mass, top = mass.cpu().numpy()[0], top.cpu().numpy()[0]
+
     rng = np.random.default_rng(1)
     for i, h in enumerate(heads):
         p = ref[i]
@@ -83,3 +91,5 @@ def test_full_size_layer_on_sampled_heads(name, heads):
         err = np.abs(O[h][rows] - Oref).max()
         rel = np.linalg.norm(O[h][rows] - Oref) / np.linalg.norm(Oref)
         assert err <= 2e-2 and rel <= 1e-2, (name, h, err, rel)
+        m_ref, t_ref, _ = orc.recall_rows(Q[0, h], K[0, h], g[h], Sg, cfg.scale, rrows[h], 0.1)
+        assert np.array_equal(top[h], t_ref) and np.allclose(mass[h], m_ref, rtol=1e-11, atol=0), (name, h)

@@ -418,3 +418,46 @@ def test_host_entry_points_match_device_path():
         streams[g].synchronize()
         plans[g].check()
     assert torch.equal(hO2, O_dev)
+
+
+@pytest.mark.parametrize("name,top_frac", [("tiny", 0.1), ("small", 0.1), ("small", 0.03)])
+def test_recall_diagnostics_match_oracle(name, top_frac):
+    """Attention mass and top-key share kept by S_c, for sampled queries, against exact fp64 logits: the integer
+    ratio must be identical (both sides form the same logit bits), the mass agrees to rounding of exp and sums."""
+    cfg = inputs.CONFIGS[name]
+    Q, K, V, dQ, dK, dV = _layer(cfg, 21)
+    plan = sb.Plan(sb.make_params(cfg))
+    sb.scope_plan(dQ, dK, plan)
+    plan.check()
+    ref = _oracle_plans(Q, K, cfg)
+    _compare_plan(plan, ref, cfg, what=("select",))
+    R = 9
+    rng = np.random.default_rng(5)
+    rows = np.stack([np.sort(rng.choice(cfg.N, R, replace=False)) for _ in range(cfg.H)]).astype(np.int32)
+    rows[0, 0], rows[-1, -1] = 0, cfg.N - 1
+    mass, top = sb.scope_recall(dQ, dK, plan, torch.from_numpy(rows[None]).cuda(), top_frac)
+    plan.check()
+    mass, top = mass.cpu().numpy()[0], top.cpu().numpy()[0]
+    for h in range(cfg.H):
+        m_ref, t_ref, _ = orc.recall_rows(Q[0, h], K[0, h], ref[h].g, ref[h].S, cfg.scale, rows[h], top_frac)
+        assert np.array_equal(top[h], t_ref), (h, top[h], t_ref)
+        assert np.allclose(mass[h], m_ref, rtol=1e-12, atol=0), (h, np.abs(mass[h] - m_ref).max())
+
+
+def test_recall_rejects_bad_rows_and_full_selection_keeps_everything():
+    cfg = inputs.CONFIGS["tiny"].replace(top_p=1.0)
+    Q, K, V, dQ, dK, dV = _layer(cfg, 22)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.H * cfg.Cq * cfg.N))
+    sb.scope_plan(dQ, dK, plan)
+    plan.check()
+    rows = torch.tensor([[[0, 5, cfg.N - 1], [3, 4, 7]]], dtype=torch.int32, device="cuda")
+    mass, top = sb.scope_recall(dQ, dK, plan, rows, 0.25)
+    plan.check()
+    assert torch.all((mass - 1.0).abs() < 1e-14) and torch.all(top == 1.0)
+    bad = rows.clone()
+    bad[0, 1, 2] = cfg.N
+    mass, top = sb.scope_recall(dQ, dK, plan, bad, 0.25)
+    status, _ = plan.status()
+    assert status == sb.SCOPE_ERR_INVALID_ARG
+    assert torch.isnan(mass[0, 1, 2]) and not torch.isnan(mass[0, 0]).any()
+    plan.reset_status()
