@@ -55,7 +55,10 @@ typedef enum {
 /* Problem statement of Algorithm 1 ("Require" line) plus layout. */
 typedef struct {
     int32_t B, H, N, d;       /* batch, heads, tokens per head, head dim (128) */
-    int32_t d_t, d_h, d_w;    /* contiguous channel ranges [T | H | W]; each > 0; sum == d */
+    int32_t d_t, d_h, d_w;    /* contiguous channel ranges [T | H | W]; each even; sum == d.  d_w (and d_h) may be 0
+                               * with Cw (Ch) = 1: the two-way and full-dimension partitions of the paper's
+                               * partition ablation (an empty range adds nothing to Eq. 6).  A random partition is
+                               * these ranges after scope_permute_channels() on Q and K */
     int32_t Cq, Ct, Ch, Cw;   /* cluster counts: queries, key ranges; 1 <= C <= min(N, 1024) */
     int32_t kmeans_iters;     /* Lloyd iterations, >= 1, fixed (no early exit) */
     float top_p;              /* rho of Eq. 7, in (0, 1]; >= 1 keeps every key */
@@ -170,6 +173,14 @@ scope_status scope_forward_host_async(const void *Q_host, const void *K_host, co
  * comparator of the benchmarks.  Asynchronous. */
 scope_status scope_dense_attn(const void *Q, const void *K, const void *V, const scope_plan_t *plan,
                               void *O, void *stream);
+
+/* Y[b, h, n, c] = X[b, h, n, perm[c]]: the same channel permutation applied to Q and to K leaves every
+ * q.k, hence Eq. 1 and Eq. 11, unchanged, and turns the contiguous ranges of scope_params into an
+ * arbitrary partition of the original channels (the randomly partitioned variant of the paper's
+ * partition ablation).  perm: HOST int32[128], a permutation of 0..127.  X, Y: DEVICE bf16 with the
+ * layout of `params`; they must not overlap.  Asynchronous. */
+scope_status scope_permute_channels(const void *X, const scope_params *params, const int32_t *perm,
+                                    void *Y, void *stream);
 
 /* Recall diagnostics of a finished plan (the quantity of the paper's recall figure, and the
  * retention-versus-oracle-recall protocol of its supplement, Section "Fine-Grained Key Selection at

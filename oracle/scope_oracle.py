@@ -194,8 +194,19 @@ def plan_head(Q, K, p) -> HeadPlan:
     assert d_t + d_h + d_w == d
     kq = kmeans(Q, 0, d, p.Cq, p.iters)
     ranges = ((0, d_t, p.Ct), (d_t, d_h, p.Ch), (d_t + d_h, d_w, p.Cw))
-    ks = [kmeans(K, ch0, D, Cn, p.iters) for ch0, D, Cn in ranges]
-    P = tuple(lut(kq.U, ch0, km.U)[0] for (ch0, _, _), km in zip(ranges, ks))
+    # A partition into fewer than three ranges (the partition ablation) leaves trailing ranges empty: one
+    # centroid of no channels, every key labelled 0, a table of zeros, i.e. no term in Eq. 6.
+    ks, P = [], []
+    for ch0, D, Cn in ranges:
+        if D == 0:
+            assert Cn == 1
+            ks.append(KMeansResult(np.zeros((1, 0), np.float32), np.zeros(N, np.int32), np.array([N], np.int32),
+                                   np.zeros(p.iters), np.full(p.iters, np.inf)))
+            P.append(np.zeros((p.Cq, 1), np.float32))
+        else:
+            ks.append(kmeans(K, ch0, D, Cn, p.iters))
+            P.append(lut(kq.U, ch0, ks[-1].U)[0])
+    P = tuple(P)
     z = tuple(km.assign for km in ks)
     t, b, k, r, S, margin = select_head(P, z, kq.counts, N, p.scale, p.top_p, p.k_fix, getattr(p, "select_mode", "online"))
     gap = min(float(kq.min_gap.min()), *(float(km.min_gap.min()) for km in ks))

@@ -31,7 +31,8 @@ EXPORTS = ["scope_plan_workspace_bytes", "scope_plan_create", "scope_plan_destro
            "scope_sparse_attn", "scope_forward", "scope_forward_host", "scope_forward_host_async", "scope_dense_attn", "scope_plan_status",
            "scope_plan_reset_status", "scope_plan_get", "scope_plan_field_bytes", "scope_plan_export",
            "scope_plan_import", "scope_status_string", "scope_kfix_from_alpha", "scope_kernel_launches",
-           "scope_kmeans_queries_static", "scope_recall_scratch_bytes", "scope_recall"]
+           "scope_kmeans_queries_static", "scope_recall_scratch_bytes", "scope_recall",
+           "scope_permute_channels"]
 
 
 class ScopeParams(C.Structure):
@@ -72,6 +73,7 @@ def lib():
         L.scope_sparse_attn.argtypes = [vp, vp, vp, vp, vp, vp]
         L.scope_dense_attn.argtypes = [vp, vp, vp, vp, vp, vp]
         L.scope_forward.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.scope_permute_channels.argtypes = [vp, vp, vp, vp, vp]
         L.scope_recall_scratch_bytes.argtypes = [vp, C.c_int32]
         L.scope_recall_scratch_bytes.restype = sz
         L.scope_recall.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_double, vp, sz, vp, vp, vp]
@@ -251,6 +253,16 @@ def scope_dense_attn(Q, K, V, plan: Plan, O=None):
     _check(lib().scope_dense_attn(_dev_ptr(Q, "Q"), _dev_ptr(K, "K"), _dev_ptr(V, "V"), plan.handle,
                                   _dev_ptr(O, "O"), C.c_void_p(_stream())), "scope_dense_attn")
     return O
+
+
+def scope_permute_channels(X, params: ScopeParams, perm, Y=None):
+    """Y[..., c] = X[..., perm[c]] (perm: a permutation of range(128))."""
+    if Y is None:
+        Y = torch.empty_like(X)
+    pa = (C.c_int32 * 128)(*[int(v) for v in perm])
+    _check(lib().scope_permute_channels(_dev_ptr(X, "X"), C.byref(params), pa, _dev_ptr(Y, "Y"), C.c_void_p(_stream())),
+           "scope_permute_channels")
+    return Y
 
 
 def scope_recall(Q, K, plan: Plan, rows: torch.Tensor, top_frac: float = 0.1):

@@ -69,7 +69,12 @@ scope_status validate(const scope_params *p)
         return SCOPE_ERR_INVALID_ARG;
     if (p->d != kHeadDim)
         return SCOPE_ERR_UNSUPPORTED;
-    if (p->d_t < 1 || p->d_h < 1 || p->d_w < 1 || p->d_t + p->d_h + p->d_w != p->d)
+    if (p->d_t < 1 || p->d_h < 0 || p->d_w < 0 || p->d_t + p->d_h + p->d_w != p->d)
+        return SCOPE_ERR_INVALID_ARG;
+    if ((p->d_t | p->d_h | p->d_w) & 1)
+        return SCOPE_ERR_UNSUPPORTED;  // rotary pairs: every range holds whole channel pairs
+    // a partition into fewer than three ranges leaves the trailing ones empty, with their single centroid
+    if ((p->d_h == 0 && p->d_w != 0) || (p->d_h == 0 && p->Ch != 1) || (p->d_w == 0 && p->Cw != 1))
         return SCOPE_ERR_INVALID_ARG;
     const int32_t cs[4] = {p->Cq, p->Ct, p->Ch, p->Cw};
     for (int c : cs) {
@@ -196,6 +201,17 @@ KmArgs k_args(const scope_plan_t *pl, const void *K)
     a.assign = nullptr;
     a.codes = pl->k_codes;
     a.x2 = pl->k_x2;
+    return a;
+}
+
+// the key ranges k-means runs on: the non-empty ones (they come first)
+KmArgs k_args_kmeans(const scope_plan_t *pl, const void *K)
+{
+    KmArgs a = k_args(pl, K);
+    const scope_params &p = pl->p;
+    a.nspaces = 1 + (p.d_h > 0) + (p.d_w > 0);
+    if (a.nspaces == 1)
+        a.single_field = 1;  // one range: its labels are the whole code word
     return a;
 }
 
@@ -349,7 +365,7 @@ scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, u
     }
     if (stages & SCOPE_STAGE_KMEANS_INIT) {
         launch_kmeans_init(q_args(pl, Q), st);
-        launch_kmeans_init(k_args(pl, K), st);
+        launch_kmeans_init(k_args_kmeans(pl, K), st);
     }
     if (stages & SCOPE_STAGE_KMEANS_Q) {
         KmArgs a = q_args(pl, Q);
@@ -361,7 +377,7 @@ scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, u
         }
     }
     if (stages & SCOPE_STAGE_KMEANS_K) {
-        KmArgs a = k_args(pl, K);
+        KmArgs a = k_args_kmeans(pl, K);
         if (!(stages & SCOPE_STAGE_KMEANS_INIT))
             launch_kmeans_norms(a, st);
         for (int it = 0; it < p.kmeans_iters; ++it) {
@@ -420,6 +436,34 @@ scope_status scope_sparse_attn(const void *Q, const void *K, const void *V, cons
                                void *stream)
 {
     return attn_common(Q, K, V, plan, O, stream, 0);
+}
+
+scope_status scope_permute_channels(const void *X, const scope_params *params, const int32_t *perm, void *Y,
+                                    void *stream)
+{
+    if (!X || !Y || !params || !perm || X == Y)
+        return SCOPE_ERR_INVALID_ARG;
+    scope_params p = *params;
+    scope_status v = validate(&p);
+    if (v != SCOPE_OK)
+        return v;
+    normalise(&p);
+    if (!aligned16(X) || !aligned16(Y))
+        return SCOPE_ERR_ALIGNMENT;
+    PermuteArgs a{};
+    bool seen[kHeadDim] = {};
+    for (int c = 0; c < kHeadDim; ++c) {
+        if (perm[c] < 0 || perm[c] >= kHeadDim || seen[perm[c]])
+            return SCOPE_ERR_INVALID_ARG;
+        seen[perm[c]] = true;
+        a.perm[c] = (uint8_t)perm[c];
+    }
+    a.X = static_cast<const bf16 *>(X);
+    a.Y = static_cast<bf16 *>(Y);
+    a.sb = p.stride_b; a.sh = p.stride_h; a.sn = p.stride_n;
+    a.B = p.B; a.H = p.H; a.N = p.N;
+    launch_permute_channels(a, static_cast<cudaStream_t>(stream));
+    return cuda_ok(cudaGetLastError());
 }
 
 size_t scope_recall_scratch_bytes(const scope_params *params, int32_t rows_per_head)

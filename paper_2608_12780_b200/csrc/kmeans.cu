@@ -228,11 +228,19 @@ __global__ void __launch_bounds__(NT) kmeans_assign_kernel(KmArgs a)
 
     // labels out
     if (tid < TM && tok0 + tid < a.N) {
-        if (a.nspaces == 1)
-            a.assign[(size_t)bh * a.N + tok0 + tid] = asg[0][tid];
-        else
-            a.codes[(size_t)bh * a.N + tok0 + tid] =
-                (uint32_t)asg[0][tid] | ((uint32_t)asg[1][tid] << kCodeBits) | ((uint32_t)asg[2][tid] << (2 * kCodeBits));
+        const size_t at = (size_t)bh * a.N + tok0 + tid;
+        if (a.single_field > 0) {
+            const int sh = (a.single_field - 1) * kCodeBits;
+            a.codes[at] = a.single_field == 1 ? (uint32_t)asg[0][tid]
+                                              : ((a.codes[at] & ~((uint32_t)kCodeMask << sh)) | ((uint32_t)asg[0][tid] << sh));
+        } else if (a.nspaces == 1) {
+            a.assign[at] = asg[0][tid];
+        } else {
+            uint32_t code = 0;
+            for (int s = 0; s < a.nspaces; ++s)
+                code |= (uint32_t)asg[s][tid] << (s * kCodeBits);
+            a.codes[at] = code;
+        }
     }
 
     // order the tile's tokens by label (rank by counting), then add each run of equal labels once
@@ -372,9 +380,9 @@ void launch_kmeans_iteration(const KmArgs &a, int32_t *status, cudaStream_t st)
     const bool simt = force && force[0] == '1';
     // the three key ranges in one launch if their codebooks fit shared and tensor memory together, else one
     // launch per range (codebooks of a few hundred centroids), else the general kernel
-    bool per_range = !simt && a.nspaces == 3 && a.codes != nullptr;
+    bool per_range = !simt && a.nspaces >= 2 && a.codes != nullptr;
     KmArgs one[3];
-    for (int m = 0; m < 3 && per_range; ++m) {
+    for (int m = 0; m < a.nspaces && per_range; ++m) {
         one[m] = a;
         one[m].nspaces = 1;
         one[m].sp[0] = a.sp[m];
@@ -386,7 +394,7 @@ void launch_kmeans_iteration(const KmArgs &a, int32_t *status, cudaStream_t st)
     if (!simt && kmeans_tc_supported(a, nullptr)) {
         launch_kmeans_assign_tc(a, status, st);
     } else if (per_range) {
-        for (int m = 0; m < 3; ++m)
+        for (int m = 0; m < a.nspaces; ++m)
             launch_kmeans_assign_tc(one[m], status, st);
     } else {
         dim3 grid((a.N + TM - 1) / TM, a.B * a.H);

@@ -71,6 +71,21 @@ __global__ void unpack_codes_kernel(const uint32_t *codes, int32_t *dst, int64_t
         dst[i] = (int32_t)((codes[i] >> sh) & kCodeMask);
 }
 
+// Y[..., c] = X[..., perm[c]] for every token row.  Attention is unchanged when Q and K get the same channel
+// permutation, and a contiguous split of the permuted channels is an arbitrary partition of the original ones
+// (the randomly partitioned variant of the paper's partition ablation).
+__global__ void __launch_bounds__(256) permute_channels_kernel(PermuteArgs a)
+{
+    const int bh = blockIdx.y, b = bh / a.H, h = bh % a.H;
+    const int64_t base = (int64_t)b * a.sb + (int64_t)h * a.sh;
+    const int64_t total = (int64_t)a.N * kHeadDim;
+    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t tok = e / kHeadDim;
+        const int c = (int)(e % kHeadDim);
+        a.Y[base + tok * a.sn + c] = a.X[base + tok * a.sn + a.perm[c]];
+    }
+}
+
 int blocks_for(int64_t n)
 {
     int64_t b = (n + 255) / 256;
@@ -97,6 +112,12 @@ void launch_check_offsets_i32(const int32_t *x, int rows, int cols, int32_t last
 void launch_pack_codes(uint32_t *codes, const int32_t *src, int64_t n, int field, int C, int32_t *status, cudaStream_t st)
 {
     pack_codes_kernel<<<blocks_for(n), 256, 0, st>>>(codes, src, n, field, C, status);
+    count_launch();
+}
+void launch_permute_channels(const PermuteArgs &a, cudaStream_t st)
+{
+    dim3 grid(blocks_for((int64_t)a.N * kHeadDim), a.B * a.H);
+    permute_channels_kernel<<<grid, 256, 0, st>>>(a);
     count_launch();
 }
 void launch_unpack_codes(const uint32_t *codes, int32_t *dst, int64_t n, int field, cudaStream_t st)

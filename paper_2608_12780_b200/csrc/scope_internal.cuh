@@ -141,4 +141,13 @@ void launch_check_offsets_i32(const int32_t *x, int rows, int cols, int32_t last
 void launch_pack_codes(uint32_t *codes, const int32_t *src, int64_t n, int field, int C, int32_t *status, cudaStream_t st);
 void launch_unpack_codes(const uint32_t *codes, int32_t *dst, int64_t n, int field, cudaStream_t st);
 
+struct PermuteArgs {
+    const bf16 *X;
+    bf16 *Y;
+    int64_t sb, sh, sn;
+    int B, H, N;
+    uint8_t perm[128];
+};
+void launch_permute_channels(const PermuteArgs &a, cudaStream_t st);
+
 }  // namespace scope

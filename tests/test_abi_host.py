@@ -60,6 +60,32 @@ def test_invalid_parameters_are_rejected(lib, field, value):
     assert lib.scope_plan_workspace_bytes(C.byref(_params(**{field: value}))) == 0
 
 
+def test_partitions_with_fewer_ranges(lib):
+    """Trailing key ranges may be empty (two-way and full-dimension partitions); an empty range has exactly one
+    centroid, empty ranges come last, and every range holds whole channel pairs."""
+    ok = lambda **kw: lib.scope_plan_workspace_bytes(C.byref(_params(**kw))) > 0
+    assert ok(d_t=72, d_h=56, d_w=0, Cw=1)
+    assert ok(d_t=128, d_h=0, d_w=0, Ch=1, Cw=1)
+    assert not ok(d_t=72, d_h=56, d_w=0)             # Cw must be 1
+    assert not ok(d_t=72, d_h=0, d_w=56, Ch=1)       # an empty range before a non-empty one
+    assert not ok(d_t=0, d_h=64, d_w=64, Ct=1)
+    h = C.c_void_p()
+    p = _params(d_t=17, d_h=55, d_w=56)
+    assert lib.scope_plan_create(C.byref(p), C.c_void_p(1 << 20), 1 << 30, None, C.byref(h)) == sb.SCOPE_ERR_UNSUPPORTED
+
+
+def test_permute_channels_rejects_bad_arguments(lib):
+    p = _params()
+    perm = (C.c_int32 * 128)(*range(128))
+    x, y = C.c_void_p(1 << 20), C.c_void_p(1 << 24)  # never dereferenced: validation fails first
+    assert lib.scope_permute_channels(None, C.byref(p), perm, y, None) == sb.SCOPE_ERR_INVALID_ARG
+    assert lib.scope_permute_channels(x, C.byref(p), perm, x, None) == sb.SCOPE_ERR_INVALID_ARG
+    perm[5] = 4  # not a permutation
+    assert lib.scope_permute_channels(x, C.byref(p), perm, y, None) == sb.SCOPE_ERR_INVALID_ARG
+    perm[5] = 128
+    assert lib.scope_permute_channels(x, C.byref(p), perm, y, None) == sb.SCOPE_ERR_INVALID_ARG
+
+
 def test_unsupported_and_alignment_codes(lib):
     h = C.c_void_p()
     ws = C.c_void_p(1 << 20)  # never dereferenced: every call below fails validation first

@@ -461,3 +461,53 @@ def test_recall_rejects_bad_rows_and_full_selection_keeps_everything():
     assert status == sb.SCOPE_ERR_INVALID_ARG
     assert torch.isnan(mass[0, 1, 2]) and not torch.isnan(mass[0, 0]).any()
     plan.reset_status()
+
+
+@pytest.mark.parametrize("split,C", [((128, 0, 0), (24, 1, 1)), ((72, 56, 0), (8, 16, 1)), ((16, 112, 0), (8, 40, 1))])
+def test_partitions_with_one_and_two_ranges(split, C):
+    """The full-dimension and two-way partitions of the partition ablation: empty trailing ranges."""
+    cfg = inputs.CONFIGS["small"].replace(H=3, split=split, Ct=C[0], Ch=C[1], Cw=C[2])
+    Q, K, V, dQ, dK, dV = _layer(inputs.CONFIGS["small"].replace(H=3), 31)
+    ref = _oracle_plans(Q, K, cfg)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.H * cfg.Cq * cfg.N))
+    O = _to_np(sb.scope_forward(dQ, dK, dV, plan))
+    plan.check()
+    g = plan.export("Q_ASSIGN")
+    z = [plan.export(f"K_CODES_{m}") for m in "THW"]
+    off, idx = plan.export("KEY_OFFSETS"), plan.export("KEY_INDICES")
+    for h in range(cfg.H):
+        assert np.array_equal(g[h], ref[h].g)
+        for m in range(3):
+            assert np.array_equal(z[m][h], ref[h].z[m]), (h, m)
+        assert np.array_equal(plan.export("TOPP_COUNT")[h], ref[h].t_c)
+        assert plan.export("K_HEAD")[h] == ref[h].k_head
+        for c in range(cfg.Cq):
+            assert np.array_equal(idx[off[h * cfg.Cq + c]: off[h * cfg.Cq + c + 1]], ref[h].S[c]), (h, c)
+        rows = np.arange(0, cfg.N, 7)
+        Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], ref[h].g, ref[h].S, cfg.scale, rows)
+        err, rel = _attn_errors(O[0, h][rows], Oref)
+        assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (h, err, rel)
+
+
+def test_random_partition_through_channel_permutation():
+    """Three ranges over randomly permuted channels: permute Q and K, plan as usual.  The permutation kernel is
+    an index copy (bit-exact), the plan matches the oracle on the permuted tensors, and the attention output
+    matches the oracle's on the ORIGINAL tensors (q.k does not see the permutation)."""
+    cfg = inputs.CONFIGS["small"].replace(H=2)
+    Q, K, V, dQ, dK, dV = _layer(cfg, 32)
+    perm = np.random.default_rng(9).permutation(128)
+    params = sb.make_params(cfg, index_capacity=cfg.H * cfg.Cq * cfg.N)
+    dQp, dKp = sb.scope_permute_channels(dQ, params, perm), sb.scope_permute_channels(dK, params, perm)
+    Qp, Kp = np.ascontiguousarray(Q[..., perm]), np.ascontiguousarray(K[..., perm])
+    assert np.array_equal(dQp.view(torch.int16).cpu().numpy().view(np.uint16), Qp)
+    assert np.array_equal(dKp.view(torch.int16).cpu().numpy().view(np.uint16), Kp)
+    plan = sb.Plan(params)
+    O = _to_np(sb.scope_forward(dQp, dKp, dV, plan))
+    plan.check()
+    ref = _oracle_plans(Qp, Kp, cfg)
+    _compare_plan(plan, ref, cfg)
+    for h in range(cfg.H):
+        rows = np.arange(0, cfg.N, 11)
+        Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], ref[h].g, ref[h].S, cfg.scale, rows)
+        err, rel = _attn_errors(O[0, h][rows], Oref)
+        assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (h, err, rel)

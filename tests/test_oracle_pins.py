@@ -442,3 +442,42 @@ def test_recall_against_sorted_softmax():
     full = orc.plan_head(Q, K, cfg.replace(top_p=1.0))
     mass, top, _ = orc.recall_rows(Q, K, full.g, full.S, cfg.scale, rows, frac)
     assert np.all(np.abs(mass - 1.0) < 1e-15) and np.all(top == 1.0)
+
+
+# ----------------------------------------------------------------------------- partition variants
+
+
+@pytest.mark.parametrize("split,C", [((128, 0, 0), (16, 1, 1)), ((72, 56, 0), (8, 8, 1))])
+def test_fewer_ranges_drop_terms_of_the_lookup_sum(split, C):
+    """Full-dimension and two-way partitions: the proxy logit is still the inner product with the
+    product-code representative, now made of one or two slices."""
+    cfg, Q, K, V = _head("tiny", seed=7)
+    cfg = cfg.replace(split=split, Ct=C[0], Ch=C[1], Cw=C[2])
+    pl = orc.plan_head(Q, K, cfg)
+    assert np.all(pl.z[2] == 0) and np.all(pl.P[2] == 0) and pl.U[2].shape == (1, 0)
+    rep = np.concatenate([pl.U[m][pl.z[m]] for m in range(3)], axis=1).astype(np.float64)  # [N, 128]
+    exact = pl.Qbar.astype(np.float64) @ rep.T
+    for c in (0, cfg.Cq - 1):
+        raw = orc.scores_row(pl.P[0][c], pl.P[1][c], pl.P[2][c], *pl.z)
+        assert np.allclose(raw, exact[c], rtol=1e-5, atol=1e-4)
+    if split[1] == 0:
+        # one range: the key clustering is plain k-means over all channels, the same routine as for the queries
+        km = orc.kmeans(K, 0, 128, C[0], cfg.iters)
+        assert np.array_equal(pl.z[0], km.assign) and np.array_equal(pl.U[0], km.U)
+    # the selection invariants hold as for three ranges
+    assert all(s.shape[0] == r for s, r in zip(pl.S, pl.r_c)) and np.all(pl.r_c >= pl.k_head)
+
+
+def test_channel_permutation_leaves_attention_unchanged_and_moves_the_partition():
+    cfg, Q, K, V = _head("tiny", seed=8)
+    perm = np.random.default_rng(3).permutation(128)
+    Qp, Kp = np.ascontiguousarray(Q[:, perm]), np.ascontiguousarray(K[:, perm])
+    rows = np.arange(0, cfg.N, 5)
+    a = orc.dense_rows(Q, K, V, cfg.scale, rows)
+    b = orc.dense_rows(Qp, Kp, V, cfg.scale, rows)
+    assert np.allclose(a, b, rtol=0, atol=1e-6)  # same products, another summation order
+    # the first range of the permuted tensors clusters the original channels perm[:d_t]
+    km = orc.kmeans(Kp, 0, cfg.split[0], cfg.Ct, cfg.iters)
+    sub = np.ascontiguousarray(np.concatenate([K[:, perm[:cfg.split[0]]], np.zeros((cfg.N, 128 - cfg.split[0]), np.uint16)], 1))
+    km2 = orc.kmeans(sub, 0, cfg.split[0], cfg.Ct, cfg.iters)
+    assert np.array_equal(km.assign, km2.assign)
