@@ -511,3 +511,47 @@ def test_random_partition_through_channel_permutation():
         Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], ref[h].g, ref[h].S, cfg.scale, rows)
         err, rel = _attn_errors(O[0, h][rows], Oref)
         assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (h, err, rel)
+
+
+@pytest.mark.parametrize("grid,C,k_fix", [
+    ((1, 1, 1), (1, 1, 1, 1), 1),          # a single token
+    ((1, 3, 43), (5, 3, 4, 6), 129),       # one token past a 128-token tile, floor = every key
+    ((1, 1, 257), (7, 2, 3, 5), 20),       # one token past a 256-row attention block
+    ((2, 25, 22), (1024, 1024, 1024, 1024), 64),  # the largest codebooks the packed code holds
+])
+def test_extreme_shapes(grid, C, k_fix):
+    cfg = inputs.ScopeConfig("edge", 2, 2, grid, (16, 56, 56), C[0], C[1], C[2], C[3], 2, 0.9, k_fix)
+    Q, K, V, dQ, dK, dV = _layer(cfg, 41)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.B * cfg.H * cfg.Cq * min(cfg.N, 400)))
+    O = _to_np(sb.scope_forward(dQ, dK, dV, plan))
+    plan.check()
+    refs = [orc.plan_layer(Q[b:b + 1], K[b:b + 1], cfg, threads=4) for b in range(cfg.B)]
+    _compare_plan(plan, refs[0] + refs[1], cfg)
+    for b in range(cfg.B):
+        for h in range(cfg.H):
+            rows = np.arange(0, cfg.N, max(1, cfg.N // 64))
+            r = refs[b][h]
+            Oref = orc.attention_rows(Q[b, h], K[b, h], V[b, h], r.g, r.S, cfg.scale, rows)
+            err, rel = _attn_errors(O[b, h][rows], Oref)
+            assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (b, h, err, rel)
+
+
+def test_identical_tokens_tie_everywhere():
+    """Every token the same vector: all centroids coincide, every distance and every proxy logit ties; the
+    lowest index must win each time (labels all 0, key sets = the first r_c keys)."""
+    cfg = inputs.CONFIGS["tiny"].replace(H=1)
+    Q, K, V = inputs.make_qkv(cfg, 5)
+    Q[:] = Q[0, 0, 0]
+    K[:] = K[0, 0, 0]
+    dQ, dK, dV = _dev(Q), _dev(K), _dev(V)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.Cq * cfg.N))
+    O = _to_np(sb.scope_forward(dQ, dK, dV, plan))
+    plan.check()
+    ref = _oracle_plans(Q, K, cfg)
+    _compare_plan(plan, ref, cfg)
+    assert np.all(plan.export("Q_ASSIGN") == 0) and np.all(plan.export("K_CODES_H") == 0)
+    r0 = int(ref[0].r_c[0])
+    assert np.array_equal(_key_sets(plan, 0, cfg.Cq)[0], np.arange(r0))
+    Oref = orc.attention_rows(Q[0, 0], K[0, 0], V[0, 0], ref[0].g, ref[0].S, cfg.scale, np.arange(cfg.N))
+    err, rel = _attn_errors(O[0, 0], Oref)
+    assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2
