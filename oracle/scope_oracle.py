@@ -244,6 +244,34 @@ def dense_rows(Q, K, V, scale: float, rows) -> np.ndarray:
     return out
 
 
+def rope3d(X, grid, split, tables) -> np.ndarray:
+    """3D rotary embedding of a [N, d] bf16 tensor whose tokens are the t-major raster of ``grid`` and whose
+    channels are the ranges ``split`` (T | H | W), the form in which the paper's method receives Q and K
+    ("after 3D RoPE").  Pair (2i, 2i+1) of range a at position p_a turns by tables[a] = (cos, sin)[p_a, i]:
+    y0 = x0 c - x1 s, y1 = x0 s + x1 c, every product and sum rounded to fp32, the result to bf16."""
+    X = _u16(X)
+    N, d = X.shape
+    Tg, Hg, Wg = grid
+    assert N == Tg * Hg * Wg and sum(split) == d
+    n = np.arange(N)
+    pos = (n // (Hg * Wg), (n // Wg) % Hg, n % Wg)
+    x = (X.astype(np.uint32) << np.uint32(16)).view(np.float32)
+    out = np.empty_like(x)
+    ch0 = 0
+    for a, dm in enumerate(split):
+        if dm == 0:
+            continue
+        c = np.asarray(tables[a][0], np.float32)[pos[a]]  # [N, dm/2]
+        s = np.asarray(tables[a][1], np.float32)[pos[a]]
+        x0, x1 = x[:, ch0:ch0 + dm:2], x[:, ch0 + 1:ch0 + dm:2]
+        out[:, ch0:ch0 + dm:2] = (x0 * c).astype(np.float32) - (x1 * s).astype(np.float32)
+        out[:, ch0 + 1:ch0 + dm:2] = (x0 * s).astype(np.float32) + (x1 * c).astype(np.float32)
+        ch0 += dm
+    u = out.view(np.uint32)
+    r = u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))  # round to nearest even (finite inputs)
+    return (r >> np.uint32(16)).astype(np.uint16)
+
+
 def recall_rows(Q, K, g, S, scale: float, rows, top_frac: float):
     """Recall diagnostics of the key set of each listed query (its cluster's S_c) against the exact logits of
     Eq. 1: (attention mass kept, share of the keys at or above the ceil(top_frac N)-th largest logit kept,

@@ -123,6 +123,18 @@ def _harmonics(grid):
     return s, c
 
 
+def rope_axis_tables(grid, split):
+    """Per-axis rotary tables for callers that rotate on the device: three (cos, sin) pairs, fp32
+    [axis length, d_axis / 2], the same values the generator rotates with."""
+    out = []
+    for dm, P in zip(split, grid):
+        i = np.arange(dm // 2, dtype=np.float64)
+        w = ROPE_THETA ** (-2.0 * i / dm) if dm else i
+        ang = np.arange(P, dtype=np.float64)[:, None] * w[None, :]
+        out.append((np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)))
+    return out
+
+
 def _qk_head(cfg: ScopeConfig, seed: int, tensor: int, b: int, h: int, harm, rope) -> np.ndarray:
     N, d = cfg.N, cfg.d
     g = _rng(seed, tensor, b, h)
@@ -135,6 +147,8 @@ def _qk_head(cfg: ScopeConfig, seed: int, tensor: int, b: int, h: int, harm, rop
         x += hs[a][:, None] * coef[a, 0][None, :]
         x += hc[a][:, None] * coef[a, 1][None, :]
     x = bf16_bits_to_f32(f32_to_bf16_bits(x))
+    if rope is None:  # the tensor before the rotary embedding
+        return f32_to_bf16_bits(x)
     cs, sn = rope
     xe, xo = x[:, 0::2], x[:, 1::2]
     out = np.empty_like(x)
@@ -148,20 +162,23 @@ def _v_head(cfg: ScopeConfig, seed: int, b: int, h: int) -> np.ndarray:
     return f32_to_bf16_bits(g.standard_normal((cfg.N, cfg.d), dtype=np.float32))
 
 
-def make_head(cfg: ScopeConfig, seed: int, b: int, h: int, _tables=None):
-    """(Q, K, V) bf16 bit patterns [N, d] of one (batch, head)."""
+def make_head(cfg: ScopeConfig, seed: int, b: int, h: int, _tables=None, pre_rope: bool = False):
+    """(Q, K, V) bf16 bit patterns [N, d] of one (batch, head); ``pre_rope`` stops before the rotary embedding."""
     harm, rope = _tables if _tables is not None else (_harmonics(cfg.grid), _rope_tables(cfg.grid, cfg.split))
+    if pre_rope:
+        rope = None
     return (_qk_head(cfg, seed, 0, b, h, harm, rope), _qk_head(cfg, seed, 1, b, h, harm, rope),
             _v_head(cfg, seed, b, h))
 
 
-def make_qkv(cfg: ScopeConfig, seed: int = 0, threads: int = 8, batch_offset: int = 0, out=None):
+def make_qkv(cfg: ScopeConfig, seed: int = 0, threads: int = 8, batch_offset: int = 0, out=None, pre_rope: bool = False):
     """(Q, K, V) uint16 arrays [B, H, N, d]; heads are generated independently.
 
     ``batch_offset`` shifts the batch index used for the random streams, so that
     several processes can each draw their own slice of one larger batch.
     ``out`` may hold three preallocated uint16 arrays (e.g. views of pinned
-    host memory).
+    host memory).  ``pre_rope`` returns Q and K as they are before the rotary
+    embedding (the same draws; V is unaffected).
     """
     B, H, N, d = cfg.B, cfg.H, cfg.N, cfg.d
     if out is None:
@@ -171,7 +188,7 @@ def make_qkv(cfg: ScopeConfig, seed: int = 0, threads: int = 8, batch_offset: in
 
     def work(bh):
         b, h = divmod(bh, H)
-        q, k, v = make_head(cfg, seed, b + batch_offset, h, tables)
+        q, k, v = make_head(cfg, seed, b + batch_offset, h, tables, pre_rope)
         Q[b, h], K[b, h], V[b, h] = q, k, v
 
     if threads <= 1:

@@ -481,3 +481,48 @@ def test_channel_permutation_leaves_attention_unchanged_and_moves_the_partition(
     sub = np.ascontiguousarray(np.concatenate([K[:, perm[:cfg.split[0]]], np.zeros((cfg.N, 128 - cfg.split[0]), np.uint16)], 1))
     km2 = orc.kmeans(sub, 0, cfg.split[0], cfg.Ct, cfg.iters)
     assert np.array_equal(km.assign, km2.assign)
+
+
+# ----------------------------------------------------------------------------- rotary embedding
+
+
+def test_rope_is_a_rotation_by_relative_position():
+    cfg = inputs.CONFIGS["tiny"]
+    tables = inputs.rope_axis_tables(cfg.grid, cfg.split)
+    Qpre, Kpre, _ = inputs.make_head(cfg, 3, 0, 0, pre_rope=True)
+    Qr, Kr = orc.rope3d(Qpre, cfg.grid, cfg.split, tables), orc.rope3d(Kpre, cfg.grid, cfg.split, tables)
+    q, k, qr, kr = (_f32(x).astype(np.float64) for x in (Qpre, Kpre, Qr, Kr))
+    # token 0 sits at position (0, 0, 0): untouched
+    assert np.array_equal(Qr[0], Qpre[0])
+    # every channel pair keeps its length (up to the two bf16 roundings)
+    pair = lambda x: x[:, 0::2] ** 2 + x[:, 1::2] ** 2
+    assert np.allclose(pair(qr), pair(q), rtol=2e-2, atol=1e-3)
+    # <R_p q, R_p' k> depends on p - p' only: two token pairs with the same offset along w (same t, h)
+    Tg, Hg, Wg = cfg.grid
+    i, j = 1 * Hg * Wg + 2 * Wg + 1, 1 * Hg * Wg + 2 * Wg + 4       # offset 3 along w
+    # build q' , k' = the SAME pre-rotation vectors placed at two other positions with the same offset
+    X = Qpre.copy(); Y = Kpre.copy()
+    i2, j2 = i + 2, j + 2
+    X[i2], Y[j2] = Qpre[i], Kpre[j]
+    Xr, Yr = orc.rope3d(X, cfg.grid, cfg.split, tables), orc.rope3d(Y, cfg.grid, cfg.split, tables)
+    a = qr[i] @ kr[j]
+    b = _f32(Xr[i2]).astype(np.float64) @ _f32(Yr[j2]).astype(np.float64)
+    assert abs(a - b) <= 2e-2 * (np.linalg.norm(q[i]) * np.linalg.norm(k[j]))
+
+
+def test_rope_matches_the_generator_and_the_closed_form():
+    """The generator rotates its own draws with separately written code: both must give the same bits; and a
+    pair (1, 0) at position p turns into (cos, sin) of the table."""
+    cfg = inputs.CONFIGS["tiny"]
+    tables = inputs.rope_axis_tables(cfg.grid, cfg.split)
+    for tensor in (0, 1):
+        pre = inputs.make_head(cfg, 4, 0, 1, pre_rope=True)[tensor]
+        post = inputs.make_head(cfg, 4, 0, 1)[tensor]
+        assert np.array_equal(orc.rope3d(pre, cfg.grid, cfg.split, tables), post)
+    X = np.zeros((cfg.N, 128), np.float32)
+    X[:, 0::2] = 1.0
+    R = _f32(orc.rope3d(_bits(X), cfg.grid, cfg.split, tables))
+    n = cfg.N - 1
+    t, h, w = n // (cfg.grid[1] * cfg.grid[2]), (n // cfg.grid[2]) % cfg.grid[1], n % cfg.grid[2]
+    assert np.allclose(R[n, 0:16:2], tables[0][0][t], atol=4e-3) and np.allclose(R[n, 1:16:2], tables[0][1][t], atol=4e-3)
+    assert np.allclose(R[n, 72::2], tables[2][0][w], atol=4e-3) and np.allclose(R[n, 73::2], tables[2][1][w], atol=4e-3)
