@@ -174,6 +174,29 @@ scope_status scope_forward_host_async(const void *Q_host, const void *K_host, co
 scope_status scope_dense_attn(const void *Q, const void *K, const void *V, const scope_plan_t *plan,
                               void *O, void *stream);
 
+/* 3D rotary embedding fused into the plan.  The paper's method receives Q and K "after 3D RoPE"; a caller
+ * that holds them BEFORE the embedding can let the first k-means pass apply it while it reads the
+ * tensors anyway, instead of a separate pass over Q and K.
+ * Token n sits at (t, h, w) with n = (t * grid_h + h) * grid_w + w; the channel pair (2i, 2i+1) of range
+ * a in {T, H, W} turns by the angle whose cosine and sine are cos_a[p_a * (d_a / 2) + i] and sin_a[...]:
+ * y0 = x0 c - x1 s, y1 = x0 s + x1 c, every product and sum rounded to fp32, the result to bf16.
+ * Tables: DEVICE float, owned by the caller; those of an empty range may be NULL. */
+typedef struct {
+    int32_t grid_t, grid_h, grid_w;   /* grid_t * grid_h * grid_w == N */
+    const float *cos_t, *sin_t;       /* [grid_t, d_t / 2] */
+    const float *cos_h, *sin_h;       /* [grid_h, d_h / 2] */
+    const float *cos_w, *sin_w;       /* [grid_w, d_w / 2] */
+    int32_t fuse;                     /* 0: rotate Q and K in a pass of their own before the plan (one read and one
+                                       * write of each); 1: inside the first k-means pass where that pass runs on the
+                                       * tensor-core kernel.  Same bits either way */
+} scope_rope;
+
+/* scope_plan() on tensors that still lack their rotary embedding.  Q and K are DEVICE bf16 with the
+ * layout of the plan and ARE WRITTEN: when the call's work on the stream is done they hold the
+ * rotated tensors (the ones scope_sparse_attn must be given), and the plan is the plan of those.
+ * Asynchronous; errors as scope_plan. */
+scope_status scope_plan_rope(void *Q, void *K, const scope_rope *rope, scope_plan_t *plan, void *stream);
+
 /* Y[b, h, n, c] = X[b, h, n, perm[c]]: the same channel permutation applied to Q and to K leaves every
  * q.k, hence Eq. 1 and Eq. 11, unchanged, and turns the contiguous ranges of scope_params into an
  * arbitrary partition of the original channels (the randomly partitioned variant of the paper's

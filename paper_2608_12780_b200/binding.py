@@ -32,7 +32,7 @@ EXPORTS = ["scope_plan_workspace_bytes", "scope_plan_create", "scope_plan_destro
            "scope_plan_reset_status", "scope_plan_get", "scope_plan_field_bytes", "scope_plan_export",
            "scope_plan_import", "scope_status_string", "scope_kfix_from_alpha", "scope_kernel_launches",
            "scope_kmeans_queries_static", "scope_recall_scratch_bytes", "scope_recall",
-           "scope_permute_channels"]
+           "scope_permute_channels", "scope_plan_rope"]
 
 
 class ScopeParams(C.Structure):
@@ -74,6 +74,7 @@ def lib():
         L.scope_dense_attn.argtypes = [vp, vp, vp, vp, vp, vp]
         L.scope_forward.argtypes = [vp, vp, vp, vp, vp, vp]
         L.scope_permute_channels.argtypes = [vp, vp, vp, vp, vp]
+        L.scope_plan_rope.argtypes = [vp, vp, vp, vp, vp]
         L.scope_recall_scratch_bytes.argtypes = [vp, C.c_int32]
         L.scope_recall_scratch_bytes.restype = sz
         L.scope_recall.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_double, vp, sz, vp, vp, vp]
@@ -253,6 +254,30 @@ def scope_dense_attn(Q, K, V, plan: Plan, O=None):
     _check(lib().scope_dense_attn(_dev_ptr(Q, "Q"), _dev_ptr(K, "K"), _dev_ptr(V, "V"), plan.handle,
                                   _dev_ptr(O, "O"), C.c_void_p(_stream())), "scope_dense_attn")
     return O
+
+
+class ScopeRope(C.Structure):
+    _fields_ = [("grid_t", C.c_int32), ("grid_h", C.c_int32), ("grid_w", C.c_int32),
+                ("cos_t", C.c_void_p), ("sin_t", C.c_void_p), ("cos_h", C.c_void_p), ("sin_h", C.c_void_p),
+                ("cos_w", C.c_void_p), ("sin_w", C.c_void_p), ("fuse", C.c_int32)]
+
+
+def scope_plan_rope(Q, K, grid, tables, plan: Plan, fuse: bool = False) -> None:
+    """scope_plan on tensors BEFORE their 3D rotary embedding; Q and K are rotated in place.  ``tables``: three
+    (cos, sin) pairs of float32 CUDA tensors [axis length, d_axis / 2] (None for an empty range).  ``fuse``: rotate
+    inside the first k-means pass instead of a pass of its own (same bits)."""
+    ptr = []
+    for pair in tables:
+        for t in pair:
+            if t is None or t.numel() == 0:
+                ptr.append(None)
+            else:
+                if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+                    raise TypeError("rotary tables: contiguous float32 CUDA tensors")
+                ptr.append(t.data_ptr())
+    r = ScopeRope(int(grid[0]), int(grid[1]), int(grid[2]), *ptr, int(bool(fuse)))
+    _check(lib().scope_plan_rope(_dev_ptr(Q, "Q"), _dev_ptr(K, "K"), C.byref(r), plan.handle, C.c_void_p(_stream())),
+           "scope_plan_rope")
 
 
 def scope_permute_channels(X, params: ScopeParams, perm, Y=None):

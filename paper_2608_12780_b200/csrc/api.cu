@@ -345,7 +345,8 @@ scope_status scope_plan_create(const scope_params *params, void *workspace, size
 
 void scope_plan_destroy(scope_plan_t *plan) { delete plan; }
 
-scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, uint32_t stages, void *stream)
+static scope_status run_stages(const void *Q, const void *K, scope_plan_t *pl, uint32_t stages, void *stream,
+                               const scope_rope *rope)
 {
     if (!pl || (stages & ~(uint32_t)SCOPE_STAGE_ALL))
         return SCOPE_ERR_INVALID_ARG;
@@ -363,12 +364,40 @@ scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, u
         if (cudaMemsetAsync(pl->status, 0, ST_WORDS * sizeof(int32_t), st) != cudaSuccess)
             return SCOPE_ERR_CUDA;
     }
+    // Tensors that still lack their rotary embedding: the tensor-core k-means kernel applies it while it reads
+    // the tensor for the first time (and the strided initialisation rotates the rows it samples); a tensor whose
+    // k-means runs on the general kernel is rotated by a pass of its own first.
+    RopeTables rq{}, rk{};
+    if (rope) {
+        RopeTables r{};
+        r.on = 1;
+        r.Hg = rope->grid_h; r.Wg = rope->grid_w;
+        r.d_t = p.d_t; r.d_h = p.d_h;
+        r.cs[0] = rope->cos_t; r.sn[0] = rope->sin_t;
+        r.cs[1] = rope->cos_h; r.sn[1] = rope->sin_h;
+        r.cs[2] = rope->cos_w; r.sn[2] = rope->sin_w;
+        rq = rk = r;
+        bf16 *Qw = static_cast<bf16 *>(const_cast<void *>(Q)), *Kw = static_cast<bf16 *>(const_cast<void *>(K));
+        if (!rope->fuse || !kmeans_uses_tensor_cores(q_args(pl, Q))) {
+            launch_rope_inplace(Qw, p.stride_b, p.stride_h, p.stride_n, p.B, p.H, p.N, r, st);
+            rq.on = 0;
+        }
+        if (!rope->fuse || !kmeans_uses_tensor_cores(k_args_kmeans(pl, K))) {
+            launch_rope_inplace(Kw, p.stride_b, p.stride_h, p.stride_n, p.B, p.H, p.N, r, st);
+            rk.on = 0;
+        }
+    }
+    auto with_rope = [](KmArgs a, const RopeTables &r) {
+        a.rope = r;
+        a.Xw = r.on ? const_cast<bf16 *>(a.X) : nullptr;
+        return a;
+    };
     if (stages & SCOPE_STAGE_KMEANS_INIT) {
-        launch_kmeans_init(q_args(pl, Q), st);
-        launch_kmeans_init(k_args_kmeans(pl, K), st);
+        launch_kmeans_init(with_rope(q_args(pl, Q), rq), st);
+        launch_kmeans_init(with_rope(k_args_kmeans(pl, K), rk), st);
     }
     if (stages & SCOPE_STAGE_KMEANS_Q) {
-        KmArgs a = q_args(pl, Q);
+        KmArgs a = with_rope(q_args(pl, Q), rq);
         if (!(stages & SCOPE_STAGE_KMEANS_INIT))
             launch_kmeans_norms(a, st);  // centroids may have been imported
         for (int it = 0; it < p.kmeans_iters; ++it) {
@@ -377,7 +406,7 @@ scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, u
         }
     }
     if (stages & SCOPE_STAGE_KMEANS_K) {
-        KmArgs a = k_args_kmeans(pl, K);
+        KmArgs a = with_rope(k_args_kmeans(pl, K), rk);
         if (!(stages & SCOPE_STAGE_KMEANS_INIT))
             launch_kmeans_norms(a, st);
         for (int it = 0; it < p.kmeans_iters; ++it) {
@@ -414,6 +443,25 @@ scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, u
         launch_group(a, st);
     }
     return cuda_ok(cudaGetLastError());
+}
+
+scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *pl, uint32_t stages, void *stream)
+{
+    return run_stages(Q, K, pl, stages, stream, nullptr);
+}
+
+scope_status scope_plan_rope(void *Q, void *K, const scope_rope *rope, scope_plan_t *pl, void *stream)
+{
+    if (!pl || !rope || !Q || !K)
+        return SCOPE_ERR_INVALID_ARG;
+    const scope_params &p = pl->p;
+    if (rope->grid_t < 1 || rope->grid_h < 1 || rope->grid_w < 1 ||
+        (int64_t)rope->grid_t * rope->grid_h * rope->grid_w != (int64_t)p.N || (rope->fuse != 0 && rope->fuse != 1))
+        return SCOPE_ERR_INVALID_ARG;
+    if (!rope->cos_t || !rope->sin_t || (p.d_h > 0 && (!rope->cos_h || !rope->sin_h)) ||
+        (p.d_w > 0 && (!rope->cos_w || !rope->sin_w)))
+        return SCOPE_ERR_INVALID_ARG;
+    return run_stages(Q, K, pl, SCOPE_STAGE_ALL, stream, rope);
 }
 
 scope_status scope_plan(const void *Q, const void *K, scope_plan_t *plan, void *stream)

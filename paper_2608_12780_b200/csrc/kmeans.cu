@@ -312,7 +312,17 @@ __global__ void __launch_bounds__(256) kmeans_finalize_kernel(KmArgs a, int mode
         int r = e / sp.D, ch = e % sp.D;
         if (mode == 1) {
             int64_t tok = ((int64_t)r * a.N) / sp.C;
-            cent[e] = __bfloat162float(Xh[tok * a.sn + sp.ch0 + ch]);
+            const int ac = sp.ch0 + ch;
+            if (a.rope.on) {  // the tensor is rotated later, by the first pass: rotate the sampled value here
+                const uint32_t w = *reinterpret_cast<const uint32_t *>(Xh + tok * a.sn + (ac & ~1));
+                int axis;
+                size_t at;
+                rope_site(a.rope, ac >> 1, (int)tok, axis, at);
+                const uint32_t y = rope_word(w, __ldg(a.rope.cs[axis] + at), __ldg(a.rope.sn[axis] + at));
+                cent[e] = __uint_as_float((ac & 1) ? (y & 0xffff0000u) : (y << 16));
+            } else {
+                cent[e] = __bfloat162float(Xh[tok * a.sn + ac]);
+            }
         } else if (mode == 0) {
             int n = counts[r];
             if (n > 0)
@@ -374,26 +384,43 @@ void launch_kmeans_norms(const KmArgs &a, cudaStream_t st)
     count_launch();
 }
 
-void launch_kmeans_iteration(const KmArgs &a, int32_t *status, cudaStream_t st)
+// The three key ranges in one launch if their codebooks fit shared and tensor memory together, else one
+// launch per range (codebooks of a few hundred centroids), else the general kernel.
+static int kmeans_dispatch(const KmArgs &a, KmArgs *one /* [3] */)
 {
     const char *force = getenv("SCOPE_KMEANS_SIMT");  // testing aid: run the general kernel
-    const bool simt = force && force[0] == '1';
-    // the three key ranges in one launch if their codebooks fit shared and tensor memory together, else one
-    // launch per range (codebooks of a few hundred centroids), else the general kernel
-    bool per_range = !simt && a.nspaces >= 2 && a.codes != nullptr;
-    KmArgs one[3];
-    for (int m = 0; m < a.nspaces && per_range; ++m) {
+    if (force && force[0] == '1')
+        return 0;
+    if (kmeans_tc_supported(a, nullptr))
+        return 1;
+    if (a.nspaces < 2 || a.codes == nullptr)
+        return 0;
+    for (int m = 0; m < a.nspaces; ++m) {
         one[m] = a;
         one[m].nspaces = 1;
         one[m].sp[0] = a.sp[m];
         one[m].single_field = m + 1;
         one[m].assign = nullptr;
         one[m].x2_ready = a.x2_ready || m > 0;  // the first launch of a call leaves the row norms for the rest
-        per_range = kmeans_tc_supported(one[m], nullptr);
+        if (!kmeans_tc_supported(one[m], nullptr))
+            return 0;
     }
-    if (!simt && kmeans_tc_supported(a, nullptr)) {
+    return 2;
+}
+
+bool kmeans_uses_tensor_cores(const KmArgs &a)
+{
+    KmArgs one[3];
+    return kmeans_dispatch(a, one) != 0;
+}
+
+void launch_kmeans_iteration(const KmArgs &a, int32_t *status, cudaStream_t st)
+{
+    KmArgs one[3];
+    const int how = kmeans_dispatch(a, one);
+    if (how == 1) {
         launch_kmeans_assign_tc(a, status, st);
-    } else if (per_range) {
+    } else if (how == 2) {
         for (int m = 0; m < a.nspaces; ++m)
             launch_kmeans_assign_tc(one[m], status, st);
     } else {

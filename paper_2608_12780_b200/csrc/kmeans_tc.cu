@@ -171,6 +171,41 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         const bool valid = tok0 + gt < a.N;
         load_x_tile(a, Xh, tok0, xbase, gt);
         cp_async_wait<0>();
+        if (a.rope.on && !a.x2_ready) {
+            // First pass over a tensor that still lacks its rotary embedding: every thread rotates the 16-byte
+            // pieces it has just copied (its own copies are complete), in shared memory and in the tensor itself;
+            // later passes, and the attention, read the rotated tensor.  The table rows of its four channel pairs
+            // are fixed per thread; the positions of a row come from three divisions.
+            const int row0 = gt >> 4, chunk = gt & 15;
+            int axis[4], half[4], idx[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int ch = 2 * (chunk * 4 + q);
+                axis[q] = ch < a.rope.d_t ? 0 : (ch < a.rope.d_t + a.rope.d_h ? 1 : 2);
+                const int c0 = axis[q] == 0 ? 0 : (axis[q] == 1 ? a.rope.d_t : a.rope.d_t + a.rope.d_h);
+                const int dm = axis[q] == 0 ? a.rope.d_t : (axis[q] == 1 ? a.rope.d_h : kHeadDim - a.rope.d_t - a.rope.d_h);
+                half[q] = dm >> 1;
+                idx[q] = (ch - c0) >> 1;
+            }
+            unsigned char *px = s_x + grp * XTILE_BYTES + (chunk >> 3) * HALF_BYTES + sw128(row0, chunk & 7);
+            bf16 *gx = a.Xw + (int64_t)b * a.sb + (int64_t)h * a.sh + (int64_t)(tok0 + row0) * a.sn + chunk * 8;
+            const int plane = a.rope.Hg * a.rope.Wg;
+            for (int i = 0; i < TM / 8 && tok0 + row0 + 8 * i < a.N; ++i) {
+                const int n = tok0 + row0 + 8 * i;
+                const int pt = n / plane, rem = n - pt * plane, ph = rem / a.rope.Wg, pw = rem - ph * a.rope.Wg;
+                uint4 v = *reinterpret_cast<uint4 *>(px + 1024 * i);
+                uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int pos = axis[q] == 0 ? pt : (axis[q] == 1 ? ph : pw);
+                    const size_t at = (size_t)pos * half[q] + idx[q];
+                    w[q] = rope_word(w[q], __ldg(a.rope.cs[axis[q]] + at), __ldg(a.rope.sn[axis[q]] + at));
+                }
+                v = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4 *>(px + 1024 * i) = v;
+                *reinterpret_cast<uint4 *>(gx + (int64_t)8 * i * a.sn) = v;
+            }
+        }
         fence_proxy_async();
         tc_fence_before();
         bar_sync(1 + grp, 128);

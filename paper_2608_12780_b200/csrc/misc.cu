@@ -86,6 +86,35 @@ __global__ void __launch_bounds__(256) permute_channels_kernel(PermuteArgs a)
     }
 }
 
+// 3D rotary embedding of a whole tensor in place (the path for tensors whose k-means does not run on the
+// tensor-core kernel, which applies it while it reads the tensor for the first time)
+__global__ void __launch_bounds__(256) rope_inplace_kernel(bf16 *X, int64_t sb, int64_t sh, int64_t sn, int H, int N,
+                                                           RopeTables r)
+{
+    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    bf16 *Xh = X + (int64_t)b * sb + (int64_t)h * sh;
+    const int64_t total = (int64_t)N * (kHeadDim / 8);
+    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int n = (int)(e / (kHeadDim / 8)), chunk = (int)(e % (kHeadDim / 8));
+        uint4 *p = reinterpret_cast<uint4 *>(Xh + (int64_t)n * sn + chunk * 8);
+        uint4 v = *p;
+        uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        const int plane = r.Hg * r.Wg;
+        const int pt = n / plane, rem = n - pt * plane, ph = rem / r.Wg, pw = rem - ph * r.Wg;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int ch = 2 * (chunk * 4 + q);
+            const int axis = ch < r.d_t ? 0 : (ch < r.d_t + r.d_h ? 1 : 2);
+            const int c0 = axis == 0 ? 0 : (axis == 1 ? r.d_t : r.d_t + r.d_h);
+            const int dm = axis == 0 ? r.d_t : (axis == 1 ? r.d_h : kHeadDim - r.d_t - r.d_h);
+            const int pos = axis == 0 ? pt : (axis == 1 ? ph : pw);
+            const size_t at = (size_t)pos * (dm >> 1) + ((ch - c0) >> 1);
+            w[q] = rope_word(w[q], __ldg(r.cs[axis] + at), __ldg(r.sn[axis] + at));
+        }
+        *p = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 int blocks_for(int64_t n)
 {
     int64_t b = (n + 255) / 256;
@@ -112,6 +141,13 @@ void launch_check_offsets_i32(const int32_t *x, int rows, int cols, int32_t last
 void launch_pack_codes(uint32_t *codes, const int32_t *src, int64_t n, int field, int C, int32_t *status, cudaStream_t st)
 {
     pack_codes_kernel<<<blocks_for(n), 256, 0, st>>>(codes, src, n, field, C, status);
+    count_launch();
+}
+void launch_rope_inplace(bf16 *X, int64_t sb, int64_t sh, int64_t sn, int B, int H, int N, const RopeTables &r,
+                         cudaStream_t st)
+{
+    dim3 grid(blocks_for((int64_t)N * (kHeadDim / 8)), B * H);
+    rope_inplace_kernel<<<grid, 256, 0, st>>>(X, sb, sh, sn, H, N, r);
     count_launch();
 }
 void launch_permute_channels(const PermuteArgs &a, cudaStream_t st)

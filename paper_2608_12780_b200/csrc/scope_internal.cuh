@@ -33,6 +33,41 @@ struct KmSpace {
     int cpad;         // C rounded up to a multiple of 16
 };
 
+// 3D rotary embedding still to be applied to a tensor (tables on the device, [axis length][d_axis / 2]).
+struct RopeTables {
+    int on;             // 0: the tensor is already rotated
+    int Hg, Wg;         // token n sits at t = n / (Hg Wg), h = (n / Wg) % Hg, w = n % Wg
+    int d_t, d_h;       // channel ranges [0, d_t) | [d_t, d_t + d_h) | the rest
+    const float *cs[3], *sn[3];
+};
+
+#ifdef __CUDACC__
+// Rotation of the channel pair (2i, 2i+1) held in one 32-bit word (low half = channel 2i): every product
+// and sum rounded to fp32, the result to bf16.
+__device__ __forceinline__ uint32_t rope_word(uint32_t w, float c, float s)
+{
+    const float x0 = __uint_as_float(w << 16), x1 = __uint_as_float(w & 0xffff0000u);
+    const float y0 = __fsub_rn(__fmul_rn(x0, c), __fmul_rn(x1, s));
+    const float y1 = __fadd_rn(__fmul_rn(x0, s), __fmul_rn(x1, c));
+    const __nv_bfloat162 v = __floats2bfloat162_rn(y0, y1);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+// which table row a channel pair of a token reads: axis of the pair, its index inside the axis, the position
+__device__ __forceinline__ void rope_site(const RopeTables &r, int pair, int n, int &axis, size_t &at)
+{
+    const int ch = 2 * pair;
+    int i, pos, half;
+    if (ch < r.d_t) {
+        axis = 0; i = pair; pos = n / (r.Hg * r.Wg); half = r.d_t >> 1;
+    } else if (ch < r.d_t + r.d_h) {
+        axis = 1; i = (ch - r.d_t) >> 1; pos = (n / r.Wg) % r.Hg; half = r.d_h >> 1;
+    } else {
+        axis = 2; i = (ch - r.d_t - r.d_h) >> 1; pos = n % r.Wg; half = (kHeadDim - r.d_t - r.d_h) >> 1;
+    }
+    at = (size_t)pos * half + i;
+}
+#endif
+
 struct KmArgs {
     const bf16 *X;
     int64_t sb, sh, sn;
@@ -44,6 +79,8 @@ struct KmArgs {
     float *x2;         // [BH, N] squared row norms, kept from the first pass to the later ones (may be null)
     int x2_ready;      // 0: this pass computes and stores them, 1: it reads them
     int single_field;  // 0: outputs as nspaces says; m + 1: a one-range launch that writes field m of the packed codes
+    RopeTables rope;   // rope.on: X is not rotated yet; the first pass of a call (x2_ready == 0) rotates it in place
+    bf16 *Xw;          // X again, writable (rope.on only)
 };
 
 // Per (head, query cluster) result of the selection stage that later kernels read.
@@ -103,6 +140,9 @@ struct AttnArgs {
 void launch_kmeans_init(const KmArgs &a, cudaStream_t st);
 void launch_kmeans_norms(const KmArgs &a, cudaStream_t st);
 void launch_kmeans_iteration(const KmArgs &a, int32_t *status, cudaStream_t st);
+bool kmeans_uses_tensor_cores(const KmArgs &a);  // which kernel launch_kmeans_iteration picks
+void launch_rope_inplace(bf16 *X, int64_t sb, int64_t sh, int64_t sn, int B, int H, int N, const RopeTables &r,
+                         cudaStream_t st);
 bool kmeans_tc_supported(const KmArgs &a, size_t *smem_bytes);
 void launch_kmeans_assign_tc(const KmArgs &a, int32_t *status, cudaStream_t st);
 void launch_lut(int BH, int Cq, int d, const float *qcent, const KmSpace *ksp /*3*/, float *const *lut,

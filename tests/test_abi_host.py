@@ -108,6 +108,8 @@ def test_null_plan_and_pointer_checks(lib):
     assert lib.scope_forward(None, None, None, None, None, None) == sb.SCOPE_ERR_INVALID_ARG
     assert lib.scope_sparse_attn(None, None, None, None, None, None) == sb.SCOPE_ERR_INVALID_ARG
     assert lib.scope_plan_status(None, None, None) == sb.SCOPE_ERR_INVALID_ARG
+    assert lib.scope_plan_rope(None, None, None, None, None) == sb.SCOPE_ERR_INVALID_ARG
+    assert lib.scope_recall(None, None, None, None, 4, 0.1, None, 0, None, None, None) == sb.SCOPE_ERR_INVALID_ARG
     assert lib.scope_plan_field_bytes(None, 0) == 0
     lib.scope_plan_destroy(None)
 

@@ -555,3 +555,43 @@ def test_identical_tokens_tie_everywhere():
     Oref = orc.attention_rows(Q[0, 0], K[0, 0], V[0, 0], ref[0].g, ref[0].S, cfg.scale, np.arange(cfg.N))
     err, rel = _attn_errors(O[0, 0], Oref)
     assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2
+
+
+def _rope_tables_dev(cfg):
+    return [tuple(torch.from_numpy(t).cuda() for t in pair) for pair in inputs.rope_axis_tables(cfg.grid, cfg.split)]
+
+
+@pytest.mark.parametrize("fuse", [False, True])
+@pytest.mark.parametrize("case", ["small", "ragged_44_42_42", "paper_codebooks", "general_kernel", "two_ranges"])
+def test_rotary_embedding_fused_into_the_plan(case, fuse, monkeypatch):
+    """Q and K handed over BEFORE their rotary embedding: afterwards they hold exactly the rotated tensors and the
+    plan is the plan of those (tensor-core k-means: rotation inside the first pass, one launch per key range for
+    large codebooks; general kernel: a pass of its own)."""
+    if case == "small":
+        cfg = inputs.CONFIGS["small"].replace(H=2)
+    elif case == "ragged_44_42_42":
+        cfg = inputs.ScopeConfig("r", 1, 2, (3, 7, 11), (44, 42, 42), 13, 5, 9, 7, 3, 0.85, 17)
+    elif case == "paper_codebooks":
+        cfg = inputs.ScopeConfig("p", 1, 1, (6, 10, 10), (16, 56, 56), 300, 333, 333, 333, 2, 0.9, 32)
+    elif case == "general_kernel":
+        cfg = inputs.CONFIGS["small"].replace(H=2)
+        monkeypatch.setenv("SCOPE_KMEANS_SIMT", "1")
+    else:
+        cfg = inputs.CONFIGS["small"].replace(H=2, split=(72, 56, 0), Cw=1)
+    Qpre, Kpre, V = inputs.make_qkv(cfg, 51, pre_rope=True)
+    Q, K, _ = inputs.make_qkv(cfg, 51)
+    assert not np.array_equal(Qpre, Q)
+    dQ, dK, dV = _dev(Qpre), _dev(Kpre), _dev(V)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.H * cfg.Cq * cfg.N))
+    sb.scope_plan_rope(dQ, dK, cfg.grid, _rope_tables_dev(cfg), plan, fuse=fuse)
+    plan.check()
+    bits = lambda t: t.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(bits(dQ), Q) and np.array_equal(bits(dK), K)
+    ref = _oracle_plans(Q, K, cfg)
+    _compare_plan(plan, ref, cfg)
+    O = _to_np(sb.scope_sparse_attn(dQ, dK, dV, plan))
+    for h in range(cfg.H):
+        rows = np.arange(0, cfg.N, 9)
+        Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], ref[h].g, ref[h].S, cfg.scale, rows)
+        err, rel = _attn_errors(O[0, h][rows], Oref)
+        assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (h, err, rel)
