@@ -69,6 +69,11 @@ typedef struct {
                                  (batch, head, query cluster) */
     int32_t select_mode;      /* SCOPE_SELECT_* below; 0 is the method of the paper */
     int32_t reserved;         /* must be 0 */
+    int32_t n_extra;          /* key ranges beyond T | H | W (0..5): the 4- and 8-way partitions of the paper's
+                               * partition ablation.  Range 3 + i holds the next d_x[i] channels (even, >= 2) and
+                               * has C_x[i] centroids; all ranges together cover d.  Needs d_h, d_w > 0; Eq. 6 adds
+                               * the terms in range order */
+    int32_t d_x[5], C_x[5];
 } scope_params;
 
 /* Key-count rules.  ONLINE is the paper's method (Eq. 8 - Eq. 10).  The other two are the variants
@@ -101,6 +106,12 @@ typedef enum {
     SCOPE_KEY_INDICES,      /* int32 [total]          S_c, ascending key index inside a cluster */
     SCOPE_Q_PERM,           /* int32 [BH, N]          tokens grouped by query cluster, ascending inside */
     SCOPE_Q_OFFSETS,        /* int32 [BH, Cq + 1]     start of cluster c in Q_PERM (per head) */
+    SCOPE_K_CENTROIDS_X0,   /* float [BH, C_x[i], d_x[i]]  codebooks of the extra ranges, i = 0..4 (five entries) */
+    SCOPE_K_CENTROIDS_X1, SCOPE_K_CENTROIDS_X2, SCOPE_K_CENTROIDS_X3, SCOPE_K_CENTROIDS_X4,
+    SCOPE_K_CODES_X0,       /* int32 [BH, N]          codes of the extra ranges */
+    SCOPE_K_CODES_X1, SCOPE_K_CODES_X2, SCOPE_K_CODES_X3, SCOPE_K_CODES_X4,
+    SCOPE_LUT_X0,           /* float [BH, Cq, C_x[i]] tables of the extra ranges */
+    SCOPE_LUT_X1, SCOPE_LUT_X2, SCOPE_LUT_X3, SCOPE_LUT_X4,
     SCOPE_FIELD_COUNT
 } scope_field;
 

@@ -13,6 +13,7 @@
  *                            line 3; nearest centroid as in Eq. 3, mean as in Eq. 2
  *   scope_oracle_lut         score table P_m of Eq. 5
  *   scope_oracle_scores_row  indexed sum of Eq. 6 (before the 1/sqrt(d) factor)
+ *   scope_oracle_scores_row_m  the same sum for a partition into M ranges (the partition ablation)
  *   scope_oracle_topp_row    descending ranking and Top-p count of Eq. 7
  *   scope_oracle_khead       Eq. 8, Eq. 9 and the counts r_c of Eq. 10
  *   scope_oracle_key_set     the set S_c of Eq. 10
@@ -406,4 +407,18 @@ int scope_oracle_recall_row(const uint16_t *q, const uint16_t *K, int64_t row_st
     free(logit);
     free(sorted);
     return 0;
+}
+
+/* Eq. 6 for a partition into M ranges (M = 1, 2, 4, 8 in the paper's partition ablation): the indexed sum
+ * raw_j = ((P_0[z_0j] + P_1[z_1j]) + P_2[z_2j]) + ..., fp32, added in range order.  P[m] is the row of
+ * table m for one query cluster, z[m] the codes of range m.  Returns the number of table reads. */
+int64_t scope_oracle_scores_row_m(const float *const *P, const int32_t *const *z, int M, int64_t N, float *raw)
+{
+    for (int64_t j = 0; j < N; ++j) {
+        float v = P[0][z[0][j]];
+        for (int m = 1; m < M; ++m)
+            v = v + P[m][z[m][j]];
+        raw[j] = v;
+    }
+    return (int64_t)M * N;
 }

@@ -31,6 +31,8 @@ def lib():
         L.scope_oracle_lut.restype = C.c_int64
         L.scope_oracle_scores_row.argtypes = [p, p, p, p, p, p, C.c_int64, p]
         L.scope_oracle_scores_row.restype = C.c_int64
+        L.scope_oracle_scores_row_m.argtypes = [p, p, C.c_int, C.c_int64, p]
+        L.scope_oracle_scores_row_m.restype = C.c_int64
         L.scope_oracle_topp_row.argtypes = [p, C.c_int64, C.c_float, C.c_double, p, p, p]
         L.scope_oracle_topp_row.restype = C.c_int
         L.scope_oracle_khead.argtypes = [p, p, C.c_int, C.c_int64, C.c_int32, p, p, p]
@@ -107,6 +109,19 @@ def scores_row(PT, PH, PW, zT, zH, zW) -> np.ndarray:
     return raw
 
 
+def scores_row_m(P_rows, z) -> np.ndarray:
+    """Eq. 6 for any number of ranges: raw_j = ((P_0[z_0j] + P_1[z_1j]) + P_2[z_2j]) + ... in fp32, range order."""
+    M = len(P_rows)
+    rows = [np.ascontiguousarray(r, np.float32) for r in P_rows]
+    zz = [np.ascontiguousarray(v, np.int32) for v in z]
+    N = zz[0].shape[0]
+    raw = np.empty(N, np.float32)
+    pp = (C.c_void_p * M)(*[r.ctypes.data for r in rows])
+    pz = (C.c_void_p * M)(*[v.ctypes.data for v in zz])
+    lib().scope_oracle_scores_row_m(pp, pz, M, N, _ptr(raw))
+    return raw
+
+
 def topp_row(raw: np.ndarray, scale: float, rho: float):
     """(ranking pi_c, Top-p count t_c, crossing margin) of Eq. 7."""
     raw = np.ascontiguousarray(raw, np.float32)
@@ -145,9 +160,9 @@ class HeadPlan:
     Qbar: np.ndarray  # [Cq, d] fp32 query centroids (Eq. 2)
     g: np.ndarray  # [N] int32 query cluster of every token
     n_c: np.ndarray  # [Cq] int32
-    U: tuple  # three [C_m, d_m] fp32 codebooks
-    z: tuple  # three [N] int32 code vectors (Eq. 3, Eq. 4)
-    P: tuple  # three [Cq, C_m] fp32 tables (Eq. 5)
+    U: tuple  # [C_m, d_m] fp32 codebooks, one per key range (three: T, H, W; more in the partition ablation)
+    z: tuple  # [N] int32 code vectors (Eq. 3, Eq. 4)
+    P: tuple  # [Cq, C_m] fp32 tables (Eq. 5)
     t_c: np.ndarray
     b_c: np.ndarray
     k_head: int
@@ -168,7 +183,7 @@ def select_head(P, z, n_c, N: int, scale: float, top_p: float, k_fix: int, mode:
     orders, t = [], np.empty(Cq, np.int32)
     margin = np.inf
     for c in range(Cq):
-        raw = scores_row(P[0][c], P[1][c], P[2][c], z[0], z[1], z[2])
+        raw = scores_row(P[0][c], P[1][c], P[2][c], z[0], z[1], z[2]) if len(P) == 3 else scores_row_m([Pm[c] for Pm in P], z)
         order, t[c], m = topp_row(raw, scale, top_p)
         orders.append(order)
         margin = min(margin, m)
@@ -191,9 +206,11 @@ def plan_head(Q, K, p) -> HeadPlan:
     Q, K = _u16(Q), _u16(K)
     N, d = Q.shape
     d_t, d_h, d_w = p.split
-    assert d_t + d_h + d_w == d
+    assert d_t + d_h + d_w + sum(dx for dx, _ in getattr(p, "extra", ())) == d
     kq = kmeans(Q, 0, d, p.Cq, p.iters)
-    ranges = ((0, d_t, p.Ct), (d_t, d_h, p.Ch), (d_t + d_h, d_w, p.Cw))
+    ranges = [(0, d_t, p.Ct), (d_t, d_h, p.Ch), (d_t + d_h, d_w, p.Cw)]
+    for dx, cx in getattr(p, "extra", ()):  # partitions into more than three ranges
+        ranges.append((ranges[-1][0] + ranges[-1][1], dx, cx))
     # A partition into fewer than three ranges (the partition ablation) leaves trailing ranges empty: one
     # centroid of no channels, every key labelled 0, a table of zeros, i.e. no term in Eq. 6.
     ks, P = [], []

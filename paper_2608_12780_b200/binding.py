@@ -20,9 +20,11 @@ LIB_PATH = os.path.join(HERE, "libscope_b200.so")
 
 FIELDS = ["Q_CENTROIDS", "K_CENTROIDS_T", "K_CENTROIDS_H", "K_CENTROIDS_W", "Q_ASSIGN", "K_CODES_T", "K_CODES_H",
           "K_CODES_W", "CLUSTER_SIZES", "LUT_T", "LUT_H", "LUT_W", "TOPP_COUNT", "BASE_COUNT", "K_HEAD",
-          "FINAL_COUNT", "KEY_OFFSETS", "KEY_INDICES", "Q_PERM", "Q_OFFSETS"]
+          "FINAL_COUNT", "KEY_OFFSETS", "KEY_INDICES", "Q_PERM", "Q_OFFSETS"] + \
+    [f"{kind}{i}" for kind in ("K_CENTROIDS_X", "K_CODES_X", "LUT_X") for i in range(5)]
 FIELD_ID = {n: i for i, n in enumerate(FIELDS)}
-_FLOAT_FIELDS = {"Q_CENTROIDS", "K_CENTROIDS_T", "K_CENTROIDS_H", "K_CENTROIDS_W", "LUT_T", "LUT_H", "LUT_W"}
+_FLOAT_FIELDS = {"Q_CENTROIDS", "K_CENTROIDS_T", "K_CENTROIDS_H", "K_CENTROIDS_W", "LUT_T", "LUT_H", "LUT_W"} | \
+    {f"{kind}{i}" for kind in ("K_CENTROIDS_X", "LUT_X") for i in range(5)}
 
 STAGE_KMEANS_INIT, STAGE_KMEANS_Q, STAGE_KMEANS_K, STAGE_LUT, STAGE_SELECT, STAGE_GROUP = 1, 2, 4, 8, 16, 32
 STAGE_ALL = 63
@@ -41,7 +43,8 @@ class ScopeParams(C.Structure):
                 ("Cq", C.c_int32), ("Ct", C.c_int32), ("Ch", C.c_int32), ("Cw", C.c_int32),
                 ("kmeans_iters", C.c_int32), ("top_p", C.c_float), ("k_fix", C.c_int32), ("scale", C.c_float),
                 ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_n", C.c_int64),
-                ("index_capacity", C.c_int64), ("select_mode", C.c_int32), ("reserved", C.c_int32)]
+                ("index_capacity", C.c_int64), ("select_mode", C.c_int32), ("reserved", C.c_int32),
+                ("n_extra", C.c_int32), ("d_x", C.c_int32 * 5), ("C_x", C.c_int32 * 5)]
 
 
 class ScopeError(RuntimeError):
@@ -130,9 +133,15 @@ def make_params(cfg, B=None, H=None, index_capacity=None, strides=(0, 0, 0), sca
     N = cfg.N
     if index_capacity is None:
         index_capacity = max(1, int(0.35 * B * H * cfg.Cq * N))
+    extra = tuple(getattr(cfg, "extra", ()))
+    if len(extra) > 5:
+        raise ValueError("at most five key ranges beyond T | H | W")
+    dx = (C.c_int32 * 5)(*[int(e[0]) for e in extra])
+    cx = (C.c_int32 * 5)(*[int(e[1]) for e in extra])
     return ScopeParams(B, H, N, cfg.d, cfg.split[0], cfg.split[1], cfg.split[2], cfg.Cq, cfg.Ct, cfg.Ch, cfg.Cw,
                        cfg.iters, cfg.top_p, cfg.k_fix, cfg.scale if scale is None else scale,
-                       strides[0], strides[1], strides[2], int(index_capacity), int(select_mode), 0)
+                       strides[0], strides[1], strides[2], int(index_capacity), int(select_mode), 0,
+                       len(extra), dx, cx)
 
 
 def _dev_ptr(t: torch.Tensor, name: str) -> int:
@@ -174,6 +183,10 @@ class Plan:
 
     def field_shape(self, name: str):
         p, BH = self.params, self.BH
+        for kind in ("K_CENTROIDS_X", "K_CODES_X", "LUT_X"):
+            if name.startswith(kind):
+                i = int(name[len(kind):])
+                return {"K_CENTROIDS_X": (BH, p.C_x[i], p.d_x[i]), "K_CODES_X": (BH, p.N), "LUT_X": (BH, p.Cq, p.C_x[i])}[kind]
         return {
             "Q_CENTROIDS": (BH, p.Cq, p.d), "K_CENTROIDS_T": (BH, p.Ct, p.d_t), "K_CENTROIDS_H": (BH, p.Ch, p.d_h),
             "K_CENTROIDS_W": (BH, p.Cw, p.d_w), "Q_ASSIGN": (BH, p.N), "K_CODES_T": (BH, p.N), "K_CODES_H": (BH, p.N),

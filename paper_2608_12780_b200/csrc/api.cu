@@ -18,21 +18,21 @@ struct scope_plan_s {
     size_t ws_bytes;
     int32_t *status;
     // plan arrays
-    float *q_cent, *k_cent[3];
+    float *q_cent, *k_cent[8];
     int32_t *q_assign;
     uint32_t *k_codes;
     int32_t *n_c;
-    float *lut[3];
+    float *lut[8];
     int32_t *t_c, *b_c, *r_c, *k_head;
     int64_t *key_offsets;
     int32_t *key_indices;
     int32_t *q_perm, *q_offsets;
     // scratch
-    float *q_unorm, *k_unorm[3], *q_u2max, *k_u2max[3];
+    float *q_unorm, *k_unorm[8], *q_u2max, *k_u2max[8];
     float *q_x2, *k_x2;  // squared row norms of Q and K, written by the first k-means pass of a call
-    bf16 *q_split, *k_split[3];
-    double *q_sums, *k_sums[3];
-    int32_t *q_counts, *k_counts[3];
+    bf16 *q_split, *k_split[8];
+    double *q_sums, *k_sums[8];
+    int32_t *q_counts, *k_counts[8];
     RowState *rows;
     uint32_t *item_code, *item_weight;
     int32_t *item_count, *cell_table;
@@ -61,6 +61,19 @@ struct Carver {
     }
 };
 
+// key ranges: T, H, W, then the extra ones
+int n_ranges(const scope_params &p) { return 3 + p.n_extra; }
+int range_dim(const scope_params &p, int m) { return m == 0 ? p.d_t : m == 1 ? p.d_h : m == 2 ? p.d_w : p.d_x[m - 3]; }
+int range_C(const scope_params &p, int m) { return m == 0 ? p.Ct : m == 1 ? p.Ch : m == 2 ? p.Cw : p.C_x[m - 3]; }
+int range_ch0(const scope_params &p, int m)
+{
+    int c = 0;
+    for (int i = 0; i < m; ++i)
+        c += range_dim(p, i);
+    return c;
+}
+int code_words(const scope_params &p) { return (n_ranges(p) + 2) / 3; }
+
 scope_status validate(const scope_params *p)
 {
     if (!p)
@@ -69,9 +82,22 @@ scope_status validate(const scope_params *p)
         return SCOPE_ERR_INVALID_ARG;
     if (p->d != kHeadDim)
         return SCOPE_ERR_UNSUPPORTED;
-    if (p->d_t < 1 || p->d_h < 0 || p->d_w < 0 || p->d_t + p->d_h + p->d_w != p->d)
+    if (p->n_extra < 0 || p->n_extra > 5)
         return SCOPE_ERR_INVALID_ARG;
-    if ((p->d_t | p->d_h | p->d_w) & 1)
+    int dsum = p->d_t + p->d_h + p->d_w, odd = p->d_t | p->d_h | p->d_w;
+    for (int i = 0; i < p->n_extra; ++i) {
+        if (p->d_x[i] < 1 || p->C_x[i] < 1 || p->C_x[i] > p->N)
+            return SCOPE_ERR_INVALID_ARG;
+        if (p->C_x[i] > kMaxClusters)
+            return SCOPE_ERR_UNSUPPORTED;
+        dsum += p->d_x[i];
+        odd |= p->d_x[i];
+    }
+    if (p->d_t < 1 || p->d_h < 0 || p->d_w < 0 || dsum != p->d)
+        return SCOPE_ERR_INVALID_ARG;
+    if (p->n_extra > 0 && (p->d_h == 0 || p->d_w == 0))
+        return SCOPE_ERR_INVALID_ARG;  // further ranges come after three non-empty ones
+    if (odd & 1)
         return SCOPE_ERR_UNSUPPORTED;  // rotary pairs: every range holds whole channel pairs
     // a partition into fewer than three ranges leaves the trailing ones empty, with their single centroid
     if ((p->d_h == 0 && p->d_w != 0) || (p->d_h == 0 && p->Ch != 1) || (p->d_w == 0 && p->Cw != 1))
@@ -111,7 +137,12 @@ void carve(scope_plan_t *pl, unsigned char *base, size_t *total)
 {
     const scope_params &p = pl->p;
     const size_t BH = (size_t)p.B * p.H, N = p.N, Cq = p.Cq;
-    const size_t C[3] = {(size_t)p.Ct, (size_t)p.Ch, (size_t)p.Cw}, D[3] = {(size_t)p.d_t, (size_t)p.d_h, (size_t)p.d_w};
+    const int M = n_ranges(p);
+    size_t C[8] = {}, D[8] = {};
+    for (int m = 0; m < M; ++m) {
+        C[m] = (size_t)range_C(p, m);
+        D[m] = (size_t)range_dim(p, m);
+    }
     Carver cv{base};
     pl->status = cv.take<int32_t>(ST_WORDS);
     pl->q_cent = cv.take<float>(BH * Cq * p.d);
@@ -120,7 +151,7 @@ void carve(scope_plan_t *pl, unsigned char *base, size_t *total)
     pl->q_sums = cv.take<double>(BH * Cq * p.d);
     pl->q_counts = cv.take<int32_t>(BH * Cq);
     pl->q_split = cv.take<bf16>(BH * 3 * ((Cq + 15) & ~(size_t)15) * p.d);
-    for (int m = 0; m < 3; ++m) {
+    for (int m = 0; m < M; ++m) {
         pl->k_cent[m] = cv.take<float>(BH * C[m] * D[m]);
         pl->k_unorm[m] = cv.take<float>(BH * C[m]);
         pl->k_u2max[m] = cv.take<float>(BH);
@@ -132,7 +163,7 @@ void carve(scope_plan_t *pl, unsigned char *base, size_t *total)
     pl->q_assign = cv.take<int32_t>(BH * N);
     pl->q_x2 = cv.take<float>(BH * N);
     pl->k_x2 = cv.take<float>(BH * N);
-    pl->k_codes = cv.take<uint32_t>(BH * N);
+    pl->k_codes = cv.take<uint32_t>(BH * N * (size_t)code_words(p));  // word w of all heads after word w - 1
     pl->n_c = cv.take<int32_t>(BH * Cq);
     pl->t_c = cv.take<int32_t>(BH * Cq);
     pl->b_c = cv.take<int32_t>(BH * Cq);
@@ -145,7 +176,7 @@ void carve(scope_plan_t *pl, unsigned char *base, size_t *total)
     {
         // code spaces up to 2^18 cells are deduplicated through a count table
         const size_t cells = C[0] * C[1] * C[2];
-        pl->cells = cells <= ((size_t)1 << 18) ? (int)cells : 0;
+        pl->cells = (cells <= ((size_t)1 << 18) && M == 3) ? (int)cells : 0;
         pl->cell_table = cv.take<int32_t>(BH * (size_t)pl->cells);
     }
     pl->key_offsets = cv.take<int64_t>(BH * Cq + 1);
@@ -215,6 +246,24 @@ KmArgs k_args_kmeans(const scope_plan_t *pl, const void *K)
     return a;
 }
 
+// one key range as a launch of its own (partitions into more than three ranges run range by range)
+KmArgs k_range_args(const scope_plan_t *pl, const void *K, int m)
+{
+    KmArgs a{};
+    const scope_params &p = pl->p;
+    a.X = static_cast<const bf16 *>(K);
+    a.sb = p.stride_b; a.sh = p.stride_h; a.sn = p.stride_n;
+    a.B = p.B; a.H = p.H; a.N = p.N;
+    a.nspaces = 1;
+    const int C = range_C(p, m);
+    a.sp[0] = KmSpace{range_ch0(p, m), range_dim(p, m), C, pl->k_cent[m], pl->k_unorm[m], pl->k_u2max[m], pl->k_sums[m],
+                      pl->k_counts[m], nullptr, pl->k_split[m], (C + 15) & ~15};
+    a.codes = pl->k_codes;
+    a.single_field = m + 1;
+    a.x2 = pl->k_x2;
+    return a;
+}
+
 AttnArgs attn_args(const scope_plan_t *pl, const void *Q, const void *K, const void *V, void *O, int dense)
 {
     const scope_params &p = pl->p;
@@ -241,7 +290,7 @@ struct FieldInfo {
     void *ptr;
     size_t elems;
     size_t elem_bytes;
-    int code_field;  // 0..2 for packed key codes, -1 otherwise
+    int code_field;  // 0..7 for packed key codes (three fields a word), -1 otherwise
 };
 
 bool field_info(const scope_plan_t *pl, scope_field f, FieldInfo *out)
@@ -270,7 +319,21 @@ bool field_info(const scope_plan_t *pl, scope_field f, FieldInfo *out)
     case SCOPE_KEY_INDICES: fi = {pl->key_indices, (size_t)p.index_capacity, 4, -1}; break;
     case SCOPE_Q_PERM: fi = {pl->q_perm, BH * N, 4, -1}; break;
     case SCOPE_Q_OFFSETS: fi = {pl->q_offsets, BH * (Cq + 1), 4, -1}; break;
-    default: return false;
+    default:
+        if (f >= SCOPE_K_CENTROIDS_X0 && f < SCOPE_FIELD_COUNT) {
+            const int kind = ((int)f - (int)SCOPE_K_CENTROIDS_X0) / 5, i = ((int)f - (int)SCOPE_K_CENTROIDS_X0) % 5;
+            if (i >= p.n_extra)
+                return false;
+            const size_t C = (size_t)p.C_x[i], D = (size_t)p.d_x[i];
+            if (kind == 0)
+                fi = {pl->k_cent[3 + i], BH * C * D, 4, -1};
+            else if (kind == 1)
+                fi = {pl->k_codes, BH * N, 4, 3 + i};
+            else
+                fi = {pl->lut[3 + i], BH * Cq * C, 4, -1};
+            break;
+        }
+        return false;
     }
     *out = fi;
     return true;
@@ -394,7 +457,12 @@ static scope_status run_stages(const void *Q, const void *K, scope_plan_t *pl, u
     };
     if (stages & SCOPE_STAGE_KMEANS_INIT) {
         launch_kmeans_init(with_rope(q_args(pl, Q), rq), st);
-        launch_kmeans_init(with_rope(k_args_kmeans(pl, K), rk), st);
+        if (p.n_extra == 0) {
+            launch_kmeans_init(with_rope(k_args_kmeans(pl, K), rk), st);
+        } else {
+            for (int m = 0; m < n_ranges(p); ++m)
+                launch_kmeans_init(k_range_args(pl, K, m), st);
+        }
     }
     if (stages & SCOPE_STAGE_KMEANS_Q) {
         KmArgs a = with_rope(q_args(pl, Q), rq);
@@ -405,7 +473,17 @@ static scope_status run_stages(const void *Q, const void *K, scope_plan_t *pl, u
             launch_kmeans_iteration(a, pl->status, st);
         }
     }
-    if (stages & SCOPE_STAGE_KMEANS_K) {
+    if ((stages & SCOPE_STAGE_KMEANS_K) && p.n_extra > 0) {
+        for (int m = 0; m < n_ranges(p); ++m)
+            if (!(stages & SCOPE_STAGE_KMEANS_INIT))
+                launch_kmeans_norms(k_range_args(pl, K, m), st);
+        for (int it = 0; it < p.kmeans_iters; ++it)
+            for (int m = 0; m < n_ranges(p); ++m) {
+                KmArgs a = k_range_args(pl, K, m);
+                a.x2_ready = it > 0 || m > 0;  // the first launch of a call leaves the row norms for the rest
+                launch_kmeans_iteration(a, pl->status, st);
+            }
+    } else if (stages & SCOPE_STAGE_KMEANS_K) {
         KmArgs a = with_rope(k_args_kmeans(pl, K), rk);
         if (!(stages & SCOPE_STAGE_KMEANS_INIT))
             launch_kmeans_norms(a, st);
@@ -415,8 +493,10 @@ static scope_status run_stages(const void *Q, const void *K, scope_plan_t *pl, u
         }
     }
     if (stages & SCOPE_STAGE_LUT) {
-        KmArgs a = k_args(pl, K);
-        launch_lut(pl->BH, p.Cq, p.d, pl->q_cent, a.sp, pl->lut, st);
+        KmSpace sp[8];
+        for (int m = 0; m < n_ranges(p); ++m)
+            sp[m] = k_range_args(pl, K, m).sp[0];
+        launch_lut(pl->BH, p.Cq, p.d, pl->q_cent, sp, n_ranges(p), pl->lut, st);
     }
     if (stages & SCOPE_STAGE_SELECT) {
         SelectArgs a{};
@@ -427,6 +507,12 @@ static scope_status run_stages(const void *Q, const void *K, scope_plan_t *pl, u
         a.item_code = pl->item_code; a.item_weight = pl->item_weight; a.item_count = pl->item_count;
         a.cell_table = pl->cell_table; a.cells = pl->cells;
         a.lutT = pl->lut[0]; a.lutH = pl->lut[1]; a.lutW = pl->lut[2];
+        a.nx = p.n_extra;
+        for (int i = 0; i < p.n_extra; ++i) {
+            a.xC[i] = p.C_x[i];
+            a.lutX[i] = pl->lut[3 + i];
+        }
+        a.codes_x = pl->k_codes + (size_t)pl->BH * p.N;
         a.n_c = pl->n_c;
         a.t_c = pl->t_c; a.b_c = pl->b_c; a.r_c = pl->r_c; a.k_head = pl->k_head;
         a.rows = pl->rows;
@@ -455,6 +541,8 @@ scope_status scope_plan_rope(void *Q, void *K, const scope_rope *rope, scope_pla
     if (!pl || !rope || !Q || !K)
         return SCOPE_ERR_INVALID_ARG;
     const scope_params &p = pl->p;
+    if (p.n_extra != 0)
+        return SCOPE_ERR_UNSUPPORTED;  // the rotary axes are the three ranges T | H | W
     if (rope->grid_t < 1 || rope->grid_h < 1 || rope->grid_w < 1 ||
         (int64_t)rope->grid_t * rope->grid_h * rope->grid_w != (int64_t)p.N || (rope->fuse != 0 && rope->fuse != 1))
         return SCOPE_ERR_INVALID_ARG;
@@ -682,7 +770,8 @@ scope_status scope_plan_export(const scope_plan_t *pl, scope_field field, void *
     }
     const void *src = fi.ptr;
     if (fi.code_field >= 0) {
-        launch_unpack_codes(pl->k_codes, pl->io_scratch, (int64_t)fi.elems, fi.code_field, st);
+        launch_unpack_codes(pl->k_codes + (size_t)(fi.code_field / 3) * fi.elems, pl->io_scratch, (int64_t)fi.elems,
+                            fi.code_field % 3, st);
         src = pl->io_scratch;
     }
     cudaError_t e = want ? cudaMemcpyAsync(host_dst, src, want, cudaMemcpyDeviceToHost, st) : cudaSuccess;
@@ -712,14 +801,13 @@ scope_status scope_plan_import(scope_plan_t *pl, scope_field field, const void *
     if (want && cudaMemcpyAsync(dst, host_src, want, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return SCOPE_ERR_CUDA;
     const int64_t n = (int64_t)(want / fi.elem_bytes);
-    const int Cm[3] = {p.Ct, p.Ch, p.Cw};
+    if (fi.code_field >= 0) {
+        launch_pack_codes(pl->k_codes + (size_t)(fi.code_field / 3) * fi.elems, pl->io_scratch, n, fi.code_field % 3,
+                          range_C(p, fi.code_field), pl->status, st);
+        return scope_plan_status(pl, stream, nullptr);
+    }
     switch (field) {
     case SCOPE_Q_ASSIGN: launch_check_range_i32(pl->q_assign, n, 0, p.Cq - 1, pl->status, st); break;
-    case SCOPE_K_CODES_T:
-    case SCOPE_K_CODES_H:
-    case SCOPE_K_CODES_W:
-        launch_pack_codes(pl->k_codes, pl->io_scratch, n, fi.code_field, Cm[fi.code_field], pl->status, st);
-        break;
     case SCOPE_CLUSTER_SIZES: launch_check_range_i32(pl->n_c, n, 0, p.N, pl->status, st); break;
     case SCOPE_TOPP_COUNT: launch_check_range_i32(pl->t_c, n, 1, p.N, pl->status, st); break;
     case SCOPE_BASE_COUNT: launch_check_range_i32(pl->b_c, n, 1, p.N, pl->status, st); break;

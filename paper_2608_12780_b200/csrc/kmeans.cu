@@ -230,9 +230,10 @@ __global__ void __launch_bounds__(NT) kmeans_assign_kernel(KmArgs a)
     if (tid < TM && tok0 + tid < a.N) {
         const size_t at = (size_t)bh * a.N + tok0 + tid;
         if (a.single_field > 0) {
-            const int sh = (a.single_field - 1) * kCodeBits;
-            a.codes[at] = a.single_field == 1 ? (uint32_t)asg[0][tid]
-                                              : ((a.codes[at] & ~((uint32_t)kCodeMask << sh)) | ((uint32_t)asg[0][tid] << sh));
+            const int f = a.single_field - 1, sh = (f % 3) * kCodeBits;
+            uint32_t *cw = a.codes + (size_t)(f / 3) * a.B * a.H * a.N;
+            cw[at] = f % 3 == 0 ? (uint32_t)asg[0][tid]
+                                : ((cw[at] & ~((uint32_t)kCodeMask << sh)) | ((uint32_t)asg[0][tid] << sh));
         } else if (a.nspaces == 1) {
             a.assign[at] = asg[0][tid];
         } else {

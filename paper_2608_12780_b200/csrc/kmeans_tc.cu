@@ -474,9 +474,10 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             const size_t at = (size_t)bh * a.N + tok0 + gt;
             if (a.single_field > 0) {
                 // one range of the keys per launch (T, then H, then W): the first rewrites the word, the others their field
-                const int sh = (a.single_field - 1) * kCodeBits;
-                a.codes[at] = a.single_field == 1 ? (uint32_t)lab[0]
-                                                  : ((a.codes[at] & ~((uint32_t)kCodeMask << sh)) | ((uint32_t)lab[0] << sh));
+                // three 10-bit fields a word; word w of all heads follows word w - 1
+                const int f = a.single_field - 1, sh = (f % 3) * kCodeBits;
+                uint32_t *cw = a.codes + (size_t)(f / 3) * a.B * a.H * a.N;
+                cw[at] = f % 3 == 0 ? (uint32_t)lab[0] : ((cw[at] & ~((uint32_t)kCodeMask << sh)) | ((uint32_t)lab[0] << sh));
             } else if (a.nspaces == 1) {
                 a.assign[at] = lab[0];
             } else {

@@ -10,9 +10,9 @@ namespace {
 struct LutArgs {
     int Cq, d;
     const float *qcent;  // [BH, Cq, d]
-    int ch0[3], D[3], C[3];
-    const float *ucent[3];  // [BH, C_m, d_m]
-    float *lut[3];          // [BH, Cq, C_m]
+    int ch0[8], D[8], C[8];
+    const float *ucent[8];  // [BH, C_m, d_m]
+    float *lut[8];          // [BH, Cq, C_m]
 };
 
 __global__ void __launch_bounds__(256) lut_kernel(LutArgs a)
@@ -33,14 +33,15 @@ __global__ void __launch_bounds__(256) lut_kernel(LutArgs a)
 
 }  // namespace
 
-void launch_lut(int BH, int Cq, int d, const float *qcent, const KmSpace *ksp, float *const *lut, cudaStream_t st)
+void launch_lut(int BH, int Cq, int d, const float *qcent, const KmSpace *ksp, int nranges, float *const *lut,
+                cudaStream_t st)
 {
     LutArgs a;
     a.Cq = Cq;
     a.d = d;
     a.qcent = qcent;
     int maxC = 1;
-    for (int m = 0; m < 3; ++m) {
+    for (int m = 0; m < nranges; ++m) {
         a.ch0[m] = ksp[m].ch0;
         a.D[m] = ksp[m].D;
         a.C[m] = ksp[m].C;
@@ -50,7 +51,7 @@ void launch_lut(int BH, int Cq, int d, const float *qcent, const KmSpace *ksp, f
     }
     int z = (Cq * maxC + 255) / 256;
     z = z < 1 ? 1 : (z > 16 ? 16 : z);
-    lut_kernel<<<dim3(BH, 3, z), 256, 0, st>>>(a);
+    lut_kernel<<<dim3(BH, nranges, z), 256, 0, st>>>(a);
     count_launch();
 }
 

@@ -102,6 +102,11 @@ struct SelectArgs {
     int32_t *item_count;     // [BH]    scratch: number of items
     int32_t *cell_table;     // [BH, cells] scratch: keys per cell of the code space (cells > 0 only)
     int cells;               // Ct*Ch*Cw if the table is used, else 0 (every key is its own item)
+    // key ranges beyond the three of the first code word (only with cells == 0: item i is key i)
+    int nx;                  // 0..5
+    int xC[5];
+    const float *lutX[5];    // [BH, Cq, xC[i]]
+    const uint32_t *codes_x; // code words 1.. : word w of key j of head bh at codes_x[((w - 1) * BH + bh) * N + j]
     const float *lutT, *lutH, *lutW;  // [BH, Cq, Cm]
     const int32_t *n_c;      // [BH, Cq]
     int32_t *t_c, *b_c, *r_c, *k_head;
@@ -145,8 +150,8 @@ void launch_rope_inplace(bf16 *X, int64_t sb, int64_t sh, int64_t sn, int B, int
                          cudaStream_t st);
 bool kmeans_tc_supported(const KmArgs &a, size_t *smem_bytes);
 void launch_kmeans_assign_tc(const KmArgs &a, int32_t *status, cudaStream_t st);
-void launch_lut(int BH, int Cq, int d, const float *qcent, const KmSpace *ksp /*3*/, float *const *lut,
-                cudaStream_t st);
+void launch_lut(int BH, int Cq, int d, const float *qcent, const KmSpace *ksp, int nranges /* <= 8 */,
+                float *const *lut, cudaStream_t st);
 void launch_select(const SelectArgs &a, cudaStream_t st);
 void launch_group(const GroupArgs &a, cudaStream_t st);
 void launch_tiles_from_offsets(const GroupArgs &a, cudaStream_t st);

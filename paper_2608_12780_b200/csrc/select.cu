@@ -41,34 +41,74 @@ __device__ __forceinline__ float key_value(uint32_t k)
 
 struct RowTables {
     const float *T, *H, *W;  // shared-memory rows of the three tables
+    const float *X;          // rows of the extra ranges' tables, back to back
 };
 
-__device__ __forceinline__ float proxy_raw(const RowTables &t, uint32_t code)
+// the code words beyond the first of one key (partitions into more than three ranges)
+struct ExtraCodes {
+    uint32_t w[2];
+};
+template <bool WIDE>
+__device__ __forceinline__ ExtraCodes extra_codes(const SelectArgs &a, int bh, int key)
+{
+    ExtraCodes x;
+    if (!WIDE) {
+        x.w[0] = x.w[1] = 0u;
+        return x;
+    }
+    x.w[0] = a.nx > 0 ? __ldg(a.codes_x + (size_t)bh * a.N + key) : 0u;
+    x.w[1] = a.nx > 3 ? __ldg(a.codes_x + ((size_t)a.BH + bh) * a.N + key) : 0u;
+    return x;
+}
+
+template <bool WIDE>
+__device__ __forceinline__ float proxy_raw(const RowTables &t, uint32_t code, const SelectArgs &a, const ExtraCodes &x)
 {
     // Eq. 6 before the 1/sqrt(d) factor, in this order
-    float a = t.T[code & kCodeMask] + t.H[(code >> kCodeBits) & kCodeMask];
-    return a + t.W[(code >> (2 * kCodeBits)) & kCodeMask];
+    float v = t.T[code & kCodeMask] + t.H[(code >> kCodeBits) & kCodeMask];
+    v = v + t.W[(code >> (2 * kCodeBits)) & kCodeMask];
+    int off = 0;
+    for (int i = 0; WIDE && i < a.nx; ++i) {  // the further ranges, in range order
+        v = v + t.X[off + ((x.w[i / 3] >> ((i % 3) * kCodeBits)) & kCodeMask)];
+        off += a.xC[i];
+    }
+    return v;
+}
+
+__device__ __forceinline__ int tables_width(const SelectArgs &a)
+{
+    int cs = a.Ct + a.Ch + a.Cw;
+    for (int i = 0; i < a.nx; ++i)
+        cs += a.xC[i];
+    return cs;
 }
 
 __device__ __forceinline__ void load_tables(const SelectArgs &a, int bh, int c0, float *lut, RowTables *rt)
 {
-    const int CS = a.Ct + a.Ch + a.Cw;
+    const int CS = tables_width(a);
     for (int e = threadIdx.x; e < R * CS; e += NT) {
         int r = e / CS, o = e % CS;
         int c = min(c0 + r, a.Cq - 1);
         float v;
-        if (o < a.Ct)
+        if (o < a.Ct) {
             v = a.lutT[((size_t)bh * a.Cq + c) * a.Ct + o];
-        else if (o < a.Ct + a.Ch)
+        } else if (o < a.Ct + a.Ch) {
             v = a.lutH[((size_t)bh * a.Cq + c) * a.Ch + (o - a.Ct)];
-        else
+        } else if (o < a.Ct + a.Ch + a.Cw) {
             v = a.lutW[((size_t)bh * a.Cq + c) * a.Cw + (o - a.Ct - a.Ch)];
+        } else {
+            int i = 0, oo = o - a.Ct - a.Ch - a.Cw;
+            while (oo >= a.xC[i])
+                oo -= a.xC[i++];
+            v = a.lutX[i][((size_t)bh * a.Cq + c) * a.xC[i] + oo];
+        }
         lut[e] = v;
     }
     for (int r = 0; r < R; ++r) {
         rt[r].T = lut + r * CS;
         rt[r].H = rt[r].T + a.Ct;
         rt[r].W = rt[r].H + a.Ch;
+        rt[r].X = rt[r].W + a.Cw;
     }
 }
 
@@ -238,6 +278,7 @@ __global__ void __launch_bounds__(256) items_from_keys_kernel(SelectArgs a)
 
 // ---------------------------------------------------------------------------------------------
 // Top-p count t_c (Eq. 7) for R query clusters of one head.
+template <bool WIDE>
 __global__ void __launch_bounds__(NT, 2) select_topp_kernel(SelectArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -273,9 +314,10 @@ __global__ void __launch_bounds__(NT, 2) select_topp_kernel(SelectArgs a)
             m[r] = 0u;
         for (int i = tid; i < nitems; i += NT) {
             uint32_t code = __ldg(icode + i);
+            const ExtraCodes xc = extra_codes<WIDE>(a, bh, i);  // with more than three ranges item i is key i
 #pragma unroll
             for (int r = 0; r < R; ++r)
-                m[r] = max(m[r], order_key(proxy_raw(lrt[r], code)));
+                m[r] = max(m[r], order_key(proxy_raw<WIDE>(lrt[r], code, a, xc)));
         }
 #pragma unroll
         for (int r = 0; r < R; ++r) {
@@ -307,9 +349,10 @@ __global__ void __launch_bounds__(NT, 2) select_topp_kernel(SelectArgs a)
         for (int i = tid; i < nitems; i += NT) {
             const uint32_t code = __ldg(icode + i);
             const uint32_t w = __ldg(iw + i);  // keys that share this composite code (and so this logit)
+            const ExtraCodes xc = extra_codes<WIDE>(a, bh, i);
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                float raw = proxy_raw(lrt[r], code);
+                float raw = proxy_raw<WIDE>(lrt[r], code, a, xc);
                 uint32_t key = order_key(raw);
                 if (lv == 0 || (key >> pshift) == pf[r]) {
                     int bin = (key >> shift) & (nb - 1);
@@ -469,6 +512,7 @@ __global__ void __launch_bounds__(1024) khead_kernel(SelectArgs a)
 
 // ---------------------------------------------------------------------------------------------
 // Key sets S_c (Eq. 10) for R query clusters of one head, ascending key index.
+template <bool WIDE>
 __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -542,11 +586,12 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
             for (int i = tid; i < nitems; i += NT) {
                 const uint32_t code = __ldg(icode + i);
                 const uint32_t w = __ldg(iw + i);
+                const ExtraCodes xc = extra_codes<WIDE>(a, bh, i);
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
                     if (!td[r])
                         continue;
-                    uint32_t key = order_key(proxy_raw(lrt[r], code));
+                    uint32_t key = order_key(proxy_raw<WIDE>(lrt[r], code, a, xc));
                     if (lv == 0 || (key >> pshift) == pf[r])
                         atomicAdd(&cnt[r * NB + ((key >> shift) & (nb - 1))], w);
                 }
@@ -587,9 +632,10 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
         bool sel[R], tie[R];
         if (j < a.N) {
             uint32_t code = __ldg(codes + j);
+            const ExtraCodes xc = extra_codes<WIDE>(a, bh, j);
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                uint32_t key = order_key(proxy_raw(lrt[r], code));
+                uint32_t key = order_key(proxy_raw<WIDE>(lrt[r], code, a, xc));
                 sel[r] = key > tk[r];
                 tie[r] = key == tk[r];
             }
@@ -645,19 +691,29 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
 
 }  // namespace
 
+static int tables_width_host(const SelectArgs &a)
+{
+    int cs = a.Ct + a.Ch + a.Cw;
+    for (int i = 0; i < a.nx; ++i)
+        cs += a.xC[i];
+    return cs;
+}
 static size_t topp_smem(const SelectArgs &a)
 {
-    return (size_t)R * NB * (sizeof(double) + sizeof(uint32_t)) + (size_t)R * (a.Ct + a.Ch + a.Cw) * sizeof(float);
+    return (size_t)R * NB * (sizeof(double) + sizeof(uint32_t)) + (size_t)R * tables_width_host(a) * sizeof(float);
 }
 static size_t emit_smem(const SelectArgs &a)
 {
-    return (size_t)R * NB * sizeof(uint32_t) + (size_t)R * (a.Ct + a.Ch + a.Cw) * sizeof(float);
+    return (size_t)R * NB * sizeof(uint32_t) + (size_t)R * tables_width_host(a) * sizeof(float);
 }
 
 void launch_select(const SelectArgs &a, cudaStream_t st)
 {
-    cudaFuncSetAttribute(select_topp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topp_smem(a));
-    cudaFuncSetAttribute(select_emit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)emit_smem(a));
+    // the kernels come in two forms: three key ranges (one code word a key), and more (partition ablation)
+    auto topp = a.nx > 0 ? select_topp_kernel<true> : select_topp_kernel<false>;
+    auto emit = a.nx > 0 ? select_emit_kernel<true> : select_emit_kernel<false>;
+    cudaFuncSetAttribute(topp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topp_smem(a));
+    cudaFuncSetAttribute(emit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)emit_smem(a));
     if (a.cells > 0) {
         cudaMemsetAsync(a.cell_table, 0, (size_t)a.BH * a.cells * sizeof(int32_t), st);
         dedupe_count_kernel<<<dim3(std::min(64, (a.N + 255) / 256), a.BH), 256, 0, st>>>(a);
@@ -667,9 +723,9 @@ void launch_select(const SelectArgs &a, cudaStream_t st)
     }
     count_launch(a.cells > 0 ? 2 : 1);
     dim3 grid((a.Cq + R - 1) / R, a.BH);
-    select_topp_kernel<<<grid, NT, topp_smem(a), st>>>(a);
+    topp<<<grid, NT, topp_smem(a), st>>>(a);
     khead_kernel<<<1, 1024, 0, st>>>(a);
-    select_emit_kernel<<<grid, NT, emit_smem(a), st>>>(a);
+    emit<<<grid, NT, emit_smem(a), st>>>(a);
     count_launch(3);
 }
 

@@ -46,6 +46,7 @@ class ScopeConfig:
     iters: int
     top_p: float
     k_fix: int
+    extra: tuple = ()  # further key ranges after T | H | W: ((channels, centroids), ...), up to five
 
     @property
     def N(self) -> int:
@@ -53,7 +54,7 @@ class ScopeConfig:
 
     @property
     def d(self) -> int:
-        return sum(self.split)
+        return sum(self.split) + sum(dx for dx, _ in self.extra)
 
     @property
     def scale(self) -> float:

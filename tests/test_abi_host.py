@@ -74,6 +74,22 @@ def test_partitions_with_fewer_ranges(lib):
     assert lib.scope_plan_create(C.byref(p), C.c_void_p(1 << 20), 1 << 30, None, C.byref(h)) == sb.SCOPE_ERR_UNSUPPORTED
 
 
+def test_partitions_with_more_ranges(lib):
+    def params(**kw):
+        p = _params(**{k: v for k, v in kw.items() if k not in ("d_x", "C_x")})
+        for k in ("d_x", "C_x"):
+            for i, v in enumerate(kw.get(k, ())):
+                getattr(p, k)[i] = v
+        return p
+    ok = lambda **kw: lib.scope_plan_workspace_bytes(C.byref(params(**kw))) > 0
+    assert ok(d_t=32, d_h=32, d_w=32, n_extra=1, d_x=(32,), C_x=(5,))
+    assert ok(d_t=16, d_h=16, d_w=16, n_extra=5, d_x=(16,) * 5, C_x=(3, 4, 5, 6, 7))
+    assert not ok(d_t=32, d_h=32, d_w=32, n_extra=1, d_x=(30,), C_x=(5,))       # channels do not add up
+    assert not ok(d_t=32, d_h=32, d_w=32, n_extra=1, d_x=(32,), C_x=(0,))
+    assert not ok(d_t=96, d_h=0, d_w=0, Ch=1, Cw=1, n_extra=1, d_x=(32,), C_x=(5,))  # extras after empty ranges
+    assert not ok(d_t=16, d_h=16, d_w=16, n_extra=6, d_x=(16,) * 5, C_x=(3,) * 5)
+
+
 def test_permute_channels_rejects_bad_arguments(lib):
     p = _params()
     perm = (C.c_int32 * 128)(*range(128))

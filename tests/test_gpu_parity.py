@@ -595,3 +595,38 @@ def test_rotary_embedding_fused_into_the_plan(case, fuse, monkeypatch):
         Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], ref[h].g, ref[h].S, cfg.scale, rows)
         err, rel = _attn_errors(O[0, h][rows], Oref)
         assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (h, err, rel)
+
+
+@pytest.mark.parametrize("M,C", [(4, 12), (8, 9), (8, 333)])
+def test_partitions_into_four_and_eight_ranges(M, C):
+    """The 4- and 8-way partitions of the partition ablation: one k-means launch per range, two or three code
+    words per key, the lookup sum over M tables in range order."""
+    dm = 128 // M
+    base = inputs.CONFIGS["small"].replace(H=2)
+    cfg = base.replace(split=(dm, dm, dm), Ct=C, Ch=C + 1, Cw=C + 2, extra=tuple((dm, C + 3 + i) for i in range(M - 3)))
+    Q, K, V, dQ, dK, dV = _layer(base, 61)
+    ref = _oracle_plans(Q, K, cfg)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.H * cfg.Cq * cfg.N))
+    O = _to_np(sb.scope_forward(dQ, dK, dV, plan))
+    plan.check()
+    names = ["T", "H", "W"] + [f"X{i}" for i in range(M - 3)]
+    off, idx = plan.export("KEY_OFFSETS"), plan.export("KEY_INDICES")
+    for m, nm in enumerate(names):
+        z, u, P = plan.export(f"K_CODES_{nm}"), plan.export(f"K_CENTROIDS_{nm}"), plan.export(f"LUT_{nm}")
+        for h in range(cfg.H):
+            assert np.array_equal(z[h], ref[h].z[m]), (nm, h)
+            assert np.array_equal(u[h], ref[h].U[m]), (nm, h)
+            assert np.array_equal(P[h], ref[h].P[m]), (nm, h)
+    for h in range(cfg.H):
+        assert np.array_equal(plan.export("Q_ASSIGN")[h], ref[h].g)
+        assert np.array_equal(plan.export("TOPP_COUNT")[h], ref[h].t_c) and plan.export("K_HEAD")[h] == ref[h].k_head
+        for c in range(cfg.Cq):
+            assert np.array_equal(idx[off[h * cfg.Cq + c]: off[h * cfg.Cq + c + 1]], ref[h].S[c]), (h, c)
+        rows = np.arange(0, cfg.N, 13)
+        Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], ref[h].g, ref[h].S, cfg.scale, rows)
+        err, rel = _attn_errors(O[0, h][rows], Oref)
+        assert err <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (h, err, rel)
+    # codes of an extra range survive an export / import round trip
+    z = plan.export(f"K_CODES_X{M - 4}")
+    plan.import_(f"K_CODES_X{M - 4}", z)
+    assert np.array_equal(plan.export(f"K_CODES_X{M - 4}"), z) and np.array_equal(plan.export("K_CODES_T")[0], ref[0].z[0])

@@ -526,3 +526,28 @@ def test_rope_matches_the_generator_and_the_closed_form():
     t, h, w = n // (cfg.grid[1] * cfg.grid[2]), (n // cfg.grid[2]) % cfg.grid[1], n % cfg.grid[2]
     assert np.allclose(R[n, 0:16:2], tables[0][0][t], atol=4e-3) and np.allclose(R[n, 1:16:2], tables[0][1][t], atol=4e-3)
     assert np.allclose(R[n, 72::2], tables[2][0][w], atol=4e-3) and np.allclose(R[n, 73::2], tables[2][1][w], atol=4e-3)
+
+
+@pytest.mark.parametrize("M", [4, 8])
+def test_partitions_into_more_ranges(M):
+    """The 4- and 8-way partitions of the partition ablation: the indexed sum over M tables is the inner product
+    with the M-slice representative, added in range order; M = 3 through the general routine reproduces the
+    three-table routine bit for bit."""
+    cfg, Q, K, V = _head("tiny", seed=9)
+    dm = 128 // M
+    cfg = cfg.replace(split=(dm, dm, dm), Ct=6, Ch=5, Cw=7, extra=tuple((dm, 4 + i) for i in range(M - 3)))
+    pl = orc.plan_head(Q, K, cfg)
+    assert len(pl.U) == M and all(u.shape[1] == dm for u in pl.U)
+    rep = np.concatenate([pl.U[m][pl.z[m]] for m in range(M)], axis=1).astype(np.float64)
+    exact = pl.Qbar.astype(np.float64) @ rep.T
+    c = 3
+    raw = orc.scores_row_m([P[c] for P in pl.P], pl.z)
+    assert np.allclose(raw, exact[c], rtol=1e-5, atol=1e-4)
+    # range order, fp32: a hand evaluation of key 0
+    v = np.float32(pl.P[0][c][pl.z[0][0]])
+    for m in range(1, M):
+        v = np.float32(v + pl.P[m][c][pl.z[m][0]])
+    assert raw[0] == v
+    three = orc.scores_row_m([P[c] for P in pl.P[:3]], pl.z[:3])
+    assert np.array_equal(three, orc.scores_row(pl.P[0][c], pl.P[1][c], pl.P[2][c], *pl.z[:3]))
+    assert all(s.shape[0] == r for s, r in zip(pl.S, pl.r_c)) and np.all(pl.r_c >= pl.k_head)
