@@ -5,7 +5,14 @@ Chains the C steps in the order of Algorithm 1 (one attention head), Algorithm 2
 Top-k selection).  Inputs are uint16 arrays of bf16 bit patterns, [N, d] per
 head.  Nothing here may be imported by the CUDA package.
 
-Parity pins: see tests/test_oracle_pins.py.
+Besides the algorithms, three things the paper refers to without printing them are restated here in numpy or C, with
+the readings taken listed beside each: the 3D rotary embedding Q and K carry on arrival (`rope3d`), the partitions of
+the partition ablation (empty trailing ranges, more than three ranges: `plan_head`, `scores_row_m`), and the recall
+diagnostics of the recall figure and the matched-recall protocol (`recall_rows`).
+
+Parity pins: every function is pinned in tests/test_oracle_pins.py (hand-worked toys, closed forms, library routines,
+a separately written Lloyd, the input generator's own rotation).  The paper prints no numeric worked example, so
+value-level parity against the paper itself is unpinned.
 """
 from __future__ import annotations
 
