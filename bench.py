@@ -126,7 +126,7 @@ def run_reference(args, cfg):
 
 
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -138,7 +138,14 @@ class ClockSampler:
         except OSError:
             self.p = None
 
+    def mark(self):
+        """The timed region starts now (the sampler itself is started before the warm-up: nvidia-smi takes a
+        few hundred milliseconds to deliver its first sample)."""
+        self.t0 = time.time()
+
     def stop(self):
+        import datetime
+        t1 = time.time()
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.p is None:
             return out
@@ -149,24 +156,28 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        sm, mx, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        rows = []  # (time, sm, max, reasons)
         for line in self.f:
             tok = [t.strip() for t in line.split(",")]
-            if len(tok) < 7:
+            if len(tok) < 8:
                 continue
             try:
-                sm.append(float(tok[0]))
-                mx.append(float(tok[1]))
+                ts = datetime.datetime.strptime(tok[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(tok[1]), float(tok[2]),
+                             {n for n, v in zip(names, tok[4:8]) if v.lower().startswith("active")}))
             except ValueError:
                 continue
-            for n, v in zip(names, tok[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
         self.f.close()
         os.unlink(self.f.name)
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        t0 = getattr(self, "t0", None)
+        inside = [r for r in rows if t0 is not None and t0 <= r[0] <= t1 + 0.05]
+        window = "timed region"
+        if len(inside) < 3:  # a short region: the warm-up steps before it ran the same work
+            inside, window = rows, "warm-up and timed region"
+        if inside:
+            out.update(sm_mhz=float(np.median([r[1] for r in inside])), sm_max_mhz=float(max(r[2] for r in inside)),
+                       reasons=sorted(set().union(*[r[3] for r in inside])), samples=len(inside), window=window)
         return out
 
 
@@ -215,6 +226,7 @@ def run_scope(args, cfg):
         if e_mid is not None:
             e_mid[1].record(stream)
 
+    sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(max(3, args.warmup)):
         step()
     need = plan.check("warm-up")
@@ -222,9 +234,10 @@ def run_scope(args, cfg):
     # ---- timed region: K steps, device-resident inputs (3 x %d MB per layer: larger than L2)
     mids = [(ev(), ev()) for _ in range(args.steps)]
     e0, e1 = ev(), ev()
-    sampler = ClockSampler(local) if rank == 0 else None
     launches0 = sb.scope_kernel_launches()
     barrier()
+    if sampler:
+        sampler.mark()
     e0.record(stream)
     for k in range(args.steps):
         step(mids[k])
