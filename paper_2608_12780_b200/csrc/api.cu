@@ -470,6 +470,7 @@ static scope_status run_stages(const void *Q, const void *K, scope_plan_t *pl, u
             launch_kmeans_norms(a, st);  // centroids may have been imported
         for (int it = 0; it < p.kmeans_iters; ++it) {
             a.x2_ready = it > 0;
+            a.incremental = it > 1;  // about a fifth of the tokens move in the second pass: summing afresh is cheaper there
             launch_kmeans_iteration(a, pl->status, st);
         }
     }
@@ -481,6 +482,7 @@ static scope_status run_stages(const void *Q, const void *K, scope_plan_t *pl, u
             for (int m = 0; m < n_ranges(p); ++m) {
                 KmArgs a = k_range_args(pl, K, m);
                 a.x2_ready = it > 0 || m > 0;  // the first launch of a call leaves the row norms for the rest
+                a.incremental = it > 1;  // about a fifth of the tokens move in the second pass: summing afresh is cheaper there
                 launch_kmeans_iteration(a, pl->status, st);
             }
     } else if (stages & SCOPE_STAGE_KMEANS_K) {
@@ -489,6 +491,7 @@ static scope_status run_stages(const void *Q, const void *K, scope_plan_t *pl, u
             launch_kmeans_norms(a, st);
         for (int it = 0; it < p.kmeans_iters; ++it) {
             a.x2_ready = it > 0;
+            a.incremental = it > 1;  // about a fifth of the tokens move in the second pass: summing afresh is cheaper there
             launch_kmeans_iteration(a, pl->status, st);
         }
     }

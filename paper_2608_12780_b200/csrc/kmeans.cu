@@ -296,8 +296,9 @@ __global__ void __launch_bounds__(NT) kmeans_assign_kernel(KmArgs a)
 }
 
 // mode 0: centroids from member sums (empty clusters keep theirs); mode 1: evenly strided tokens;
-// mode 2: centroids as they are (imported).  All refresh the squared norms and clear the sums for
-// the next iteration.
+// mode 2: centroids as they are (imported).  All refresh the squared norms.  The member sums and counts are
+// left alone: a full pass starts from zeroed totals (launch_kmeans_iteration clears them), an incremental one
+// from the totals of the pass before.
 __global__ void __launch_bounds__(256) kmeans_finalize_kernel(KmArgs a, int mode)
 {
     __shared__ float red[256];
@@ -308,47 +309,52 @@ __global__ void __launch_bounds__(256) kmeans_finalize_kernel(KmArgs a, int mode
     float *cent = sp.cent + (size_t)bh * sp.C * sp.D;
     double *sums = sp.sums + (size_t)bh * sp.C * sp.D;
     int32_t *counts = sp.counts + (size_t)bh * sp.C;
+    // the block owns a slab of (padded) centroid rows; only the largest squared norm crosses blocks (atomic max
+    // on the bits of a non-negative float, into a word the launcher has cleared)
+    const int rpb = (sp.cpad + gridDim.z - 1) / gridDim.z;
+    const int r0 = blockIdx.z * rpb, r1 = min(sp.cpad, r0 + rpb), rc1 = min(sp.C, r1);
 
-    for (int e = threadIdx.x; e < sp.C * sp.D; e += blockDim.x) {
-        int r = e / sp.D, ch = e % sp.D;
+    for (int e = threadIdx.x; e < (rc1 - r0) * sp.D; e += blockDim.x) {
+        const int r = r0 + e / sp.D, ch = e % sp.D;
+        const size_t at = (size_t)r * sp.D + ch;
         if (mode == 1) {
             int64_t tok = ((int64_t)r * a.N) / sp.C;
             const int ac = sp.ch0 + ch;
             if (a.rope.on) {  // the tensor is rotated later, by the first pass: rotate the sampled value here
                 const uint32_t w = *reinterpret_cast<const uint32_t *>(Xh + tok * a.sn + (ac & ~1));
                 int axis;
-                size_t at;
-                rope_site(a.rope, ac >> 1, (int)tok, axis, at);
-                const uint32_t y = rope_word(w, __ldg(a.rope.cs[axis] + at), __ldg(a.rope.sn[axis] + at));
-                cent[e] = __uint_as_float((ac & 1) ? (y & 0xffff0000u) : (y << 16));
+                size_t tat;
+                rope_site(a.rope, ac >> 1, (int)tok, axis, tat);
+                const uint32_t y = rope_word(w, __ldg(a.rope.cs[axis] + tat), __ldg(a.rope.sn[axis] + tat));
+                cent[at] = __uint_as_float((ac & 1) ? (y & 0xffff0000u) : (y << 16));
             } else {
-                cent[e] = __bfloat162float(Xh[tok * a.sn + ac]);
+                cent[at] = __bfloat162float(Xh[tok * a.sn + ac]);
             }
         } else if (mode == 0) {
             int n = counts[r];
             if (n > 0)
-                cent[e] = (float)(sums[e] / (double)n);
+                cent[at] = (float)(sums[at] / (double)n);
         }
-        sums[e] = 0.0;
     }
     __syncthreads();
     if (sp.split) {
         // u = hi + mid + lo in bf16 (exact to 24 bits), laid out over absolute channels
         bf16 *split = sp.split + (size_t)bh * 3 * sp.cpad * kHeadDim;
-        for (int e = threadIdx.x; e < sp.cpad * kHeadDim; e += blockDim.x) {
-            int r = e / kHeadDim, ch = e % kHeadDim;
+        for (int e = threadIdx.x; e < (r1 - r0) * kHeadDim; e += blockDim.x) {
+            const int r = r0 + e / kHeadDim, ch = e % kHeadDim;
+            const size_t at = (size_t)r * kHeadDim + ch;
             float u = (r < sp.C && ch >= sp.ch0 && ch < sp.ch0 + sp.D) ? cent[(size_t)r * sp.D + (ch - sp.ch0)] : 0.f;
             bf16 hi = __float2bfloat16_rn(u);
-            float r1 = u - __bfloat162float(hi);
-            bf16 mid = __float2bfloat16_rn(r1);
-            bf16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
-            split[e] = hi;
-            split[(size_t)sp.cpad * kHeadDim + e] = mid;
-            split[(size_t)2 * sp.cpad * kHeadDim + e] = lo;
+            float r1f = u - __bfloat162float(hi);
+            bf16 mid = __float2bfloat16_rn(r1f);
+            bf16 lo = __float2bfloat16_rn(r1f - __bfloat162float(mid));
+            split[at] = hi;
+            split[(size_t)sp.cpad * kHeadDim + at] = mid;
+            split[(size_t)2 * sp.cpad * kHeadDim + at] = lo;
         }
     }
     float mx = 0.f;
-    for (int r = threadIdx.x; r < sp.C; r += blockDim.x) {
+    for (int r = r0 + threadIdx.x; r < rc1; r += blockDim.x) {
         float n2 = 0.f;
         for (int ch = 0; ch < sp.D; ++ch)
             n2 = fmaf(cent[(size_t)r * sp.D + ch], cent[(size_t)r * sp.D + ch], n2);
@@ -356,7 +362,6 @@ __global__ void __launch_bounds__(256) kmeans_finalize_kernel(KmArgs a, int mode
         mx = fmaxf(mx, n2);
         if (mode == 0 && sp.sizes)
             sp.sizes[(size_t)bh * sp.C + r] = counts[r];
-        counts[r] = 0;
     }
     red[threadIdx.x] = mx;
     __syncthreads();
@@ -366,23 +371,32 @@ __global__ void __launch_bounds__(256) kmeans_finalize_kernel(KmArgs a, int mode
         __syncthreads();
     }
     if (threadIdx.x == 0)
-        sp.u2max[bh] = red[0];
+        atomicMax(reinterpret_cast<int *>(sp.u2max + bh), __float_as_int(red[0]));
+}
+
+// slabs of 16 rows per block, at most 16 blocks a codebook
+static void launch_finalize(const KmArgs &a, int mode, cudaStream_t st)
+{
+    int z = 1;
+    for (int s = 0; s < a.nspaces; ++s) {
+        cudaMemsetAsync(a.sp[s].u2max, 0, (size_t)a.B * a.H * sizeof(float), st);
+        z = max(z, min(16, (a.sp[s].cpad + 15) / 16));
+    }
+    dim3 grid(a.B * a.H, a.nspaces, z);
+    kmeans_finalize_kernel<<<grid, 256, 0, st>>>(a, mode);
+    count_launch();
 }
 
 }  // namespace
 
 void launch_kmeans_init(const KmArgs &a, cudaStream_t st)
 {
-    dim3 grid(a.B * a.H, a.nspaces);
-    kmeans_finalize_kernel<<<grid, 256, 0, st>>>(a, 1);
-    count_launch();
+    launch_finalize(a, 1, st);
 }
 
 void launch_kmeans_norms(const KmArgs &a, cudaStream_t st)
 {
-    dim3 grid(a.B * a.H, a.nspaces);
-    kmeans_finalize_kernel<<<grid, 256, 0, st>>>(a, 2);
-    count_launch();
+    launch_finalize(a, 2, st);
 }
 
 // The three key ranges in one launch if their codebooks fit shared and tensor memory together, else one
@@ -415,10 +429,20 @@ bool kmeans_uses_tensor_cores(const KmArgs &a)
     return kmeans_dispatch(a, one) != 0;
 }
 
-void launch_kmeans_iteration(const KmArgs &a, int32_t *status, cudaStream_t st)
+void launch_kmeans_iteration(const KmArgs &a_in, int32_t *status, cudaStream_t st)
 {
+    KmArgs a = a_in;
     KmArgs one[3];
-    const int how = kmeans_dispatch(a, one);
+    int how = kmeans_dispatch(a, one);
+    if (how == 0)
+        a.incremental = 0;  // the general kernel sums every token in every pass
+    if (!a.incremental) {
+        for (int s = 0; s < a.nspaces; ++s) {
+            const size_t n = (size_t)a.B * a.H * a.sp[s].C;
+            cudaMemsetAsync(a.sp[s].sums, 0, n * a.sp[s].D * sizeof(double), st);
+            cudaMemsetAsync(a.sp[s].counts, 0, n * sizeof(int32_t), st);
+        }
+    }
     if (how == 1) {
         launch_kmeans_assign_tc(a, status, st);
     } else if (how == 2) {
@@ -429,9 +453,7 @@ void launch_kmeans_iteration(const KmArgs &a, int32_t *status, cudaStream_t st)
         kmeans_assign_kernel<<<grid, NT, 0, st>>>(a);
         count_launch();
     }
-    dim3 fgrid(a.B * a.H, a.nspaces);
-    kmeans_finalize_kernel<<<fgrid, 256, 0, st>>>(a, 0);
-    count_launch();
+    launch_finalize(a, 0, st);
 }
 
 }  // namespace scope

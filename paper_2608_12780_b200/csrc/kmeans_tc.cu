@@ -214,6 +214,8 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             tc_fence_after();
             G.nflagged = 0;
             G.ncand = 0;
+            if (a.incremental)
+                G.nruns[0] = G.nruns[1] = G.nruns[2] = 0;  // moved tokens per range
             for (int s = 0; s < a.nspaces; ++s) {
                 const int cp = L.cpad[s];
                 const int k_lo = a.sp[s].ch0 >> 4, k_hi = (a.sp[s].ch0 + a.sp[s].D + 15) >> 4;
@@ -237,6 +239,13 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             G.cnt[e] = 0u;
         // squared norm of the whole row (an upper bound of every range's slice, used in the tolerance): taken
         // from the tile in the first pass of a call and kept in global memory for the later ones
+        // the label word of the pass before (incremental passes compare against it): asked for early, used late
+        uint32_t old_word = 0u;
+        if (a.incremental && valid) {
+            const size_t at = (size_t)bh * a.N + tok0 + gt;
+            old_word = a.single_field > 0 ? __ldg(a.codes + (size_t)((a.single_field - 1) / 3) * a.B * a.H * a.N + at)
+                                          : (a.nspaces == 1 ? (uint32_t)__ldg(a.assign + at) : __ldg(a.codes + at));
+        }
         float x2 = 0.f;
         if (a.x2 != nullptr && a.x2_ready) {
             if (valid)
@@ -463,26 +472,79 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         }
         bar_sync(1 + grp, 128);
 
-        // ---- labels out, and the tile's tokens grouped by label (counting sort in shared memory)
+        // ---- labels out.  A full pass groups the tile's tokens by label (counting sort in shared memory) and sums
+        // the members of every label present; an incremental pass lists the tokens whose label changed.
         int lab[3] = {0, 0, 0}, pos[3] = {0, 0, 0};
         if (valid) {
-            for (int s = 0; s < a.nspaces; ++s) {
-                lab[s] = G.asg[s][gt];
-                const int sh = (lab[s] & 3) * 8;
-                pos[s] = (int)((atomicAdd(&G.cnt[(L.un_off[s] + lab[s]) >> 2], 1u << sh) >> sh) & 0xffu);
-            }
             const size_t at = (size_t)bh * a.N + tok0 + gt;
+            for (int s = 0; s < a.nspaces; ++s)
+                lab[s] = G.asg[s][gt];
+            int old[3] = {lab[0], lab[1], lab[2]};
             if (a.single_field > 0) {
-                // one range of the keys per launch (T, then H, then W): the first rewrites the word, the others their field
-                // three 10-bit fields a word; word w of all heads follows word w - 1
+                // one range of the keys per launch (T, then H, then W, ...): three 10-bit fields a word; word w of all
+                // heads follows word w - 1.  The first pass over field 0 rewrites the word, every other one its field.
                 const int f = a.single_field - 1, sh = (f % 3) * kCodeBits;
                 uint32_t *cw = a.codes + (size_t)(f / 3) * a.B * a.H * a.N;
-                cw[at] = f % 3 == 0 ? (uint32_t)lab[0] : ((cw[at] & ~((uint32_t)kCodeMask << sh)) | ((uint32_t)lab[0] << sh));
+                const uint32_t w = a.incremental ? old_word : (f % 3 == 0 ? 0u : cw[at]);
+                old[0] = (int)((w >> sh) & kCodeMask);
+                cw[at] = (w & ~((uint32_t)kCodeMask << sh)) | ((uint32_t)lab[0] << sh);
             } else if (a.nspaces == 1) {
+                if (a.incremental)
+                    old[0] = (int)old_word;
                 a.assign[at] = lab[0];
             } else {
+                if (a.incremental) {
+                    for (int s = 0; s < a.nspaces; ++s)
+                        old[s] = (int)((old_word >> (s * kCodeBits)) & kCodeMask);
+                }
                 a.codes[at] = (uint32_t)lab[0] | ((uint32_t)lab[1] << kCodeBits) | ((uint32_t)lab[2] << (2 * kCodeBits));
             }
+            for (int s = 0; s < a.nspaces; ++s) {
+                if (a.incremental) {
+                    if (old[s] != lab[s])  // token | old label << 7 | new label << 17
+                        G.runs[s][atomicAdd(&G.nruns[s], 1)] = (uint32_t)gt | ((uint32_t)old[s] << 7) | ((uint32_t)lab[s] << 17);
+                } else {
+                    const int sh = (lab[s] & 3) * 8;
+                    pos[s] = (int)((atomicAdd(&G.cnt[(L.un_off[s] + lab[s]) >> 2], 1u << sh) >> sh) & 0xffu);
+                }
+            }
+        }
+        if (a.incremental) {
+            bar_sync(1 + grp, 128);
+            // member totals follow the moved tokens: + x to the new label, - x to the old one (fp64 sums of bf16
+            // values are exact, so the totals equal a fresh summation); a thread owns two adjacent channels
+            const int ch = 2 * (gt & 63), hf = gt >> 6;
+            int s = 0;
+            while (s + 1 < a.nspaces && ch >= a.sp[s].ch0 + a.sp[s].D)
+                ++s;
+            const KmSpace &sp = a.sp[s];
+            const int rel = ch - sp.ch0;
+            if (rel >= 0 && rel < sp.D) {
+                double *sums = sp.sums + (size_t)bh * sp.C * sp.D + rel;
+                int32_t *counts = sp.counts + (size_t)bh * sp.C;
+                const uint32_t xpair = xbase + (ch >> 6) * HALF_BYTES + (ch & 7) * 2;
+                const uint32_t cbits = (uint32_t)((ch & 63) >> 3) << 4;
+                const int nm = G.nruns[s];
+                for (int e = hf; e < nm; e += 2) {
+                    const uint32_t mv = G.runs[s][e];
+                    const int lt = mv & 127, from = (mv >> 7) & 1023, to = mv >> 17;
+                    const uint32_t w = lds32(xpair + (sw128(lt, 0) ^ cbits));
+                    const double lo = (double)__uint_as_float(w << 16), hi = (double)__uint_as_float(w & 0xffff0000u);
+                    atomicAdd(sums + (size_t)to * sp.D, lo);
+                    atomicAdd(sums + (size_t)to * sp.D + 1, hi);
+                    atomicAdd(sums + (size_t)from * sp.D, -lo);
+                    atomicAdd(sums + (size_t)from * sp.D + 1, -hi);
+                    if (rel == 0) {
+                        atomicAdd(counts + to, 1);
+                        atomicSub(counts + from, 1);
+                    }
+                }
+            }
+            if (gt == 0)
+                G.next_tile = atomicAdd(&s_queue, 1);
+            tc_fence_before();
+            bar_sync(1 + grp, 128);  // the X tile and the label arrays are reused by the next tile
+            continue;
         }
         bar_sync(1 + grp, 128);
         if (gw < a.nspaces) {

@@ -78,6 +78,8 @@ struct KmArgs {
     uint32_t *codes;   // [BH, N] packed labels (nspaces == 3)
     float *x2;         // [BH, N] squared row norms, kept from the first pass to the later ones (may be null)
     int x2_ready;      // 0: this pass computes and stores them, 1: it reads them
+    int incremental;   // 1: sums and counts hold the previous pass's member totals and assign / codes its labels;
+                       //    the pass moves the tokens whose label changed instead of summing every token again
     int single_field;  // 0: outputs as nspaces says; m + 1: a one-range launch that writes field m of the packed codes
     RopeTables rope;   // rope.on: X is not rotated yet; the first pass of a call (x2_ready == 0) rotates it in place
     bf16 *Xw;          // X again, writable (rope.on only)
