@@ -47,6 +47,7 @@ struct Barriers {
     uint64_t s_full[QT][2];
     uint64_t p_full[QT][2];  // per S buffer, like s_full: a waiter can never fall two phases behind
     uint64_t pv_done[QT];
+    uint64_t o_done[QT];  // every P V of the query tile has been executed: O is final (used once)
 };
 
 // bounded wait (about a second of SM clock) that also gives up when another role has already failed
@@ -155,6 +156,7 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
             mbar_init(&bars.p_full[i][0], BM);
             mbar_init(&bars.p_full[i][1], BM);
             mbar_init(&bars.pv_done[i], 1);
+            mbar_init(&bars.o_done[i], 1);
         }
         mbar_fence_init();
     }
@@ -286,6 +288,8 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
                 mma_commit(&bars.pv_done[i]);
                 mma_commit(&bars.kv_empty[t % STAGES]);
             }
+            if (alive)
+                mma_commit(&bars.o_done[i]);
         }
     } else if (warp >= 5 && warp < 13 && (warp - 5) >> 2 < nact) {
         // ============ softmax + correction + epilogue: one thread per query row ============
@@ -382,15 +386,11 @@ __global__ void __launch_bounds__(NT, 1) sparse_attn_kernel(AttnArgs a, int32_t 
             tc_fence_before();
             mbar_arrive(&bars.p_full[qt][t & 1]);
         }
-        // A parity wait is only meaningful one phase back.  Waits on pv_done are skipped whenever no
-        // rescale is needed, so catch up one phase at a time: S of the last tile being complete implies
-        // the P V of tile ntiles-3 is, i.e. the barrier is at most two phases behind here.
-        if (alive && ntiles >= 2) {
-            alive = wait(&bars.pv_done[qt], (uint32_t)((ntiles - 2) & 1), abort_flag);
-            alive = __all_sync(0xffffffffu, alive);
-        }
+        // O is final when the last P V has been executed.  This has a barrier of its own: pv_done is polled only when
+        // a rescale needs it, so by now it may be any number of phases ahead of this thread, and a parity wait is
+        // only meaningful one phase back (a thread that got here late would wait for a phase that never ends).
         if (alive) {
-            alive = wait(&bars.pv_done[qt], (uint32_t)((ntiles - 1) & 1), abort_flag);
+            alive = wait(&bars.o_done[qt], 0u, abort_flag);
             alive = __all_sync(0xffffffffu, alive);
         }
         if (alive) {
