@@ -630,3 +630,29 @@ def test_partitions_into_four_and_eight_ranges(M, C):
     z = plan.export(f"K_CODES_X{M - 4}")
     plan.import_(f"K_CODES_X{M - 4}", z)
     assert np.array_equal(plan.export(f"K_CODES_X{M - 4}"), z) and np.array_equal(plan.export("K_CODES_T")[0], ref[0].z[0])
+
+
+def test_concurrent_plans_on_many_streams():
+    """Several plans of different shapes running at once on streams of their own (their blocks share SMs with each
+    other's small kernels, which moves every intra-block timing): no status but OK, and every output equal to the
+    one the same plan gives alone."""
+    shapes = [inputs.CONFIGS["W480"].replace(H=1), inputs.CONFIGS["small"].replace(H=4),
+              inputs.CONFIGS["W480"].replace(H=2, Cq=64, k_fix=128)]
+    jobs = []
+    for n, cfg in enumerate(shapes * 3):
+        Q, K, V = inputs.make_qkv(cfg, 70 + n % 3, threads=8)
+        dQ, dK, dV = _dev(Q), _dev(K), _dev(V)
+        plan = sb.Plan(sb.make_params(cfg))
+        alone = sb.scope_forward(dQ, dK, dV, plan).clone()
+        plan.check()
+        jobs.append((dQ, dK, dV, plan, alone, torch.empty_like(dQ), torch.cuda.Stream()))
+    torch.cuda.synchronize()
+    for rep in range(6):
+        for k, (dQ, dK, dV, plan, alone, out, stream) in enumerate(jobs):
+            with torch.cuda.stream(stream):
+                for _ in range(1 + (k + rep) % 3):  # streams drift apart: different kernels meet each time
+                    sb.scope_forward(dQ, dK, dV, plan, out)
+        torch.cuda.synchronize()
+        for dQ, dK, dV, plan, alone, out, stream in jobs:
+            plan.check(f"repetition {rep}")
+            assert torch.equal(out, alone)
