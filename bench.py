@@ -415,7 +415,7 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--gen-threads", type=int, default=min(16, os.cpu_count() or 1))
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--e2e-groups", type=int, default=4, help="head groups (plans / streams) of the host path")
+    ap.add_argument("--e2e-groups", type=int, default=8, help="head groups (plans / streams) of the host path")
     ap.add_argument("--dense-heads", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--recall-rows", type=int, default=8, help="sampled queries per head for the recall diagnostics (0: skip)")
