@@ -24,6 +24,7 @@ namespace {
 constexpr int R = 4;          // query clusters (rows) per block: they share every code read
 constexpr int NT = 512;       // threads per block
 constexpr int NWARP = NT / 32;
+constexpr int SUB = 4;        // sub-chunks of NT keys per block-wide prefix in the emission
 constexpr int NB = 2048;      // bins per level
 constexpr int LEVELS = 3;
 __device__ __constant__ int kShift[LEVELS] = {21, 10, 0};
@@ -221,13 +222,14 @@ __global__ void __launch_bounds__(256) dedupe_count_kernel(SelectArgs a)
         atomicAdd(table + code_cell(__ldg(codes + j), a.Ch, a.Cw), 1);
 }
 
-// one block per head: the non-empty cells in cell order -> (code, weight) items
+// one block per head: the non-empty cells in cell order -> (code, weight) items; each such cell is left holding
+// the index of its item
 __global__ void __launch_bounds__(1024) dedupe_compact_kernel(SelectArgs a)
 {
     __shared__ int wsum[32];
     __shared__ int carry;
     const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int32_t *table = a.cell_table + (size_t)bh * a.cells;
+    int32_t *table = a.cell_table + (size_t)bh * a.cells;
     uint32_t *icode = a.item_code + (size_t)bh * a.N;
     uint32_t *iw = a.item_weight + (size_t)bh * a.N;
     if (tid == 0)
@@ -248,6 +250,7 @@ __global__ void __launch_bounds__(1024) dedupe_compact_kernel(SelectArgs a)
             const int zw = cell % a.Cw, zh = (cell / a.Cw) % a.Ch, zt = cell / (a.Cw * a.Ch);
             icode[slot] = (uint32_t)zt | ((uint32_t)zh << kCodeBits) | ((uint32_t)zw << (2 * kCodeBits));
             iw[slot] = (uint32_t)n;
+            table[cell] = slot;  // the count has been taken: the cell now names its item (read by the emission)
         }
         __syncthreads();
         if (tid == 0) {
@@ -523,7 +526,7 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
     __shared__ int todo[R];       // 1: rank descent still needed
     __shared__ uint32_t prefix[R];
     __shared__ int64_t carried[R];
-    __shared__ int wsel[R][NWARP], wtie[R][NWARP];
+    __shared__ int wsel[R][SUB * NWARP], wtie[R][SUB * NWARP];
     __shared__ int base_sel[R], base_tie[R];
 
     if (a.status[ST_CODE] != 0)
@@ -627,62 +630,109 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
         nd[r] = need[r];
         off[r] = c0 + r < a.Cq ? a.key_offsets[(size_t)bh * a.Cq + c0 + r] : 0;
     }
-    for (int j0 = 0; j0 < a.N; j0 += NT) {
-        const int j = j0 + tid;
-        bool sel[R], tie[R];
-        if (j < a.N) {
-            uint32_t code = __ldg(codes + j);
-            const ExtraCodes xc = extra_codes<WIDE>(a, bh, j);
+    // With a code-count table the verdicts (above the threshold / in the threshold group, per row) are taken once
+    // per distinct code and kept in the shared memory the descents no longer need; a key then looks its item up
+    // through its cell instead of evaluating four proxy logits.
+    uint8_t *verdict = reinterpret_cast<uint8_t *>(cnt);
+    const bool by_item = !WIDE && a.cells > 0 && nitems <= R * NB * (int)sizeof(uint32_t);
+    const int32_t *cell_item = a.cell_table + (size_t)bh * a.cells;
+    if (by_item) {
+        __syncthreads();  // the descents are done with cnt
+        for (int i = tid; i < nitems; i += NT) {
+            const uint32_t code = __ldg(icode + i);
+            const ExtraCodes xc = extra_codes<WIDE>(a, bh, i);
+            uint32_t v = 0u;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                uint32_t key = order_key(proxy_raw<WIDE>(lrt[r], code, a, xc));
-                sel[r] = key > tk[r];
-                tie[r] = key == tk[r];
+                const uint32_t key = order_key(proxy_raw<WIDE>(lrt[r], code, a, xc));
+                v |= (key > tk[r] ? 1u : 0u) << r;
+                v |= (key == tk[r] ? 1u : 0u) << (R + r);
             }
-        } else {
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-                sel[r] = tie[r] = false;
+            verdict[i] = (uint8_t)v;
         }
-        uint32_t bs[R], bt[R];
+        __syncthreads();
+    }
+    // Keys are taken SUB x NT at a time: sub-chunk q holds the keys j0 + q NT + tid, so the order of the keys is
+    // (q, warp, lane); one block-wide prefix per group of sub-chunks gives every warp its first output slot.
+    for (int j0 = 0; j0 < a.N; j0 += SUB * NT) {
+        uint32_t code[SUB];
+        int item[SUB];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            bs[r] = __ballot_sync(0xffffffffu, sel[r]);
-            bt[r] = __ballot_sync(0xffffffffu, tie[r]);
-            if (lane == 0) {
-                wsel[r][warp] = __popc(bs[r]);
-                wtie[r][warp] = __popc(bt[r]);
+        for (int q = 0; q < SUB; ++q) {
+            const int j = j0 + q * NT + tid;
+            code[q] = j < a.N ? __ldg(codes + j) : 0u;
+        }
+        if (by_item) {
+#pragma unroll
+            for (int q = 0; q < SUB; ++q)
+                item[q] = j0 + q * NT + tid < a.N ? __ldg(cell_item + code_cell(code[q], a.Ch, a.Cw)) : 0;
+        }
+        uint32_t bs[SUB][R], bt[SUB][R];
+        uint32_t mine = 0u;  // this thread's verdicts: sub-chunk q in byte q (bit r: above, bit R + r: threshold group)
+#pragma unroll
+        for (int q = 0; q < SUB; ++q) {
+            const int j = j0 + q * NT + tid;
+            uint32_t v = 0u;
+            if (j < a.N && by_item) {
+                v = verdict[item[q]];
+            } else if (j < a.N) {
+                const ExtraCodes xc = extra_codes<WIDE>(a, bh, j);
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const uint32_t key = order_key(proxy_raw<WIDE>(lrt[r], code[q], a, xc));
+                    v |= (key > tk[r] ? 1u : 0u) << r;
+                    v |= (key == tk[r] ? 1u : 0u) << (R + r);
+                }
+            }
+            mine |= v << (8 * q);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                bs[q][r] = __ballot_sync(0xffffffffu, (v >> r) & 1u);
+                bt[q][r] = __ballot_sync(0xffffffffu, (v >> (R + r)) & 1u);
+                if (lane == 0) {
+                    wsel[r][q * NWARP + warp] = __popc(bs[q][r]);
+                    wtie[r][q * NWARP + warp] = __popc(bt[q][r]);
+                }
             }
         }
         __syncthreads();
-        // exclusive prefix over warps: warp (2r + q) scans row r, quantity q
+        // exclusive prefix over (sub-chunk, warp): warp (2r + k) scans row r, quantity k; two entries a lane
         if (warp < 2 * R) {
-            int r = warp >> 1, q = warp & 1;
-            int *arr = q ? wtie[r] : wsel[r];
-            int v = lane < NWARP ? arr[lane] : 0;
-            int inc = v;
+            const int r = warp >> 1, k = warp & 1;
+            int *arr = k ? wtie[r] : wsel[r];
+            static_assert(SUB * NWARP == 64, "two entries per lane");
+            const int v0 = arr[2 * lane], v1 = arr[2 * lane + 1];
+            int inc = v0 + v1;
             for (int o = 1; o < 32; o <<= 1) {
                 int u = __shfl_up_sync(0xffffffffu, inc, o);
                 if (lane >= o)
                     inc += u;
             }
-            int *base = q ? &base_tie[r] : &base_sel[r];
-            int b = *base;
+            int *base = k ? &base_tie[r] : &base_sel[r];
+            const int b = *base;
             __syncwarp();
-            if (lane < NWARP)
-                arr[lane] = b + inc - v;
+            arr[2 * lane] = b + inc - v0 - v1;
+            arr[2 * lane + 1] = b + inc - v1;
             if (lane == 31)
                 *base = b + inc;
         }
         __syncthreads();
         const uint32_t lt = (1u << lane) - 1u;
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            if (sel[r] || tie[r]) {
-                int sb = wsel[r][warp] + __popc(bs[r] & lt);
-                int tb = wtie[r][warp] + __popc(bt[r] & lt);
-                if (sel[r] || tb < nd[r])
-                    a.key_indices[off[r] + sb + min(tb, nd[r])] = j;
+        for (int q = 0; q < SUB; ++q) {
+            const uint32_t v = (mine >> (8 * q)) & 0xffu;
+            if (v == 0u)
+                continue;
+            const int j = j0 + q * NT + tid;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const bool sl = (v >> r) & 1u, ti = (v >> (R + r)) & 1u;
+                if (sl || ti) {
+                    const int sb = wsel[r][q * NWARP + warp] + __popc(bs[q][r] & lt);
+                    const int tb = wtie[r][q * NWARP + warp] + __popc(bt[q][r] & lt);
+                    if (sl || tb < nd[r])
+                        a.key_indices[off[r] + sb + min(tb, nd[r])] = j;
+                }
             }
         }
         __syncthreads();
