@@ -636,7 +636,7 @@ def test_concurrent_plans_on_many_streams():
     """Several plans of different shapes running at once on streams of their own (their blocks share SMs with each
     other's small kernels, which moves every intra-block timing): no status but OK, and every output equal to the
     one the same plan gives alone."""
-    shapes = [inputs.CONFIGS["W480"].replace(H=1), inputs.CONFIGS["small"].replace(H=4),
+    shapes = [inputs.CONFIGS["W720"].replace(H=1), inputs.CONFIGS["small"].replace(H=4),
               inputs.CONFIGS["W480"].replace(H=2, Cq=64, k_fix=128)]
     jobs = []
     for n, cfg in enumerate(shapes * 3):
@@ -647,7 +647,7 @@ def test_concurrent_plans_on_many_streams():
         plan.check()
         jobs.append((dQ, dK, dV, plan, alone, torch.empty_like(dQ), torch.cuda.Stream()))
     torch.cuda.synchronize()
-    for rep in range(6):
+    for rep in range(24):
         for k, (dQ, dK, dV, plan, alone, out, stream) in enumerate(jobs):
             with torch.cuda.stream(stream):
                 for _ in range(1 + (k + rep) % 3):  # streams drift apart: different kernels meet each time
