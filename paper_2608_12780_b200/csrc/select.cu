@@ -401,6 +401,7 @@ __global__ void __launch_bounds__(NT, 2) select_topp_kernel(SelectArgs a)
             if (lane == 0) {
                 carried_mass[r] += w_above;
                 carried_cnt[r] += c_above;
+                bin = bin < 0 ? 0 : bin;  // no crossing at all: only with non-finite masses
                 prefix[r] = (prefix[r] << kBits[lv]) | (uint32_t)bin;
                 if (lv == LEVELS - 1 && c0 + r < a.Cq) {
                     // threshold group: m keys of equal logit e_tau each; smallest i with mass_above + i e >= target
@@ -417,6 +418,7 @@ __global__ void __launch_bounds__(NT, 2) select_topp_kernel(SelectArgs a)
                     int64_t t = carried_cnt[r] + (int64_t)i;
                     if (a.top_p >= 1.0f)
                         t = a.N;
+                    t = t < 1 ? 1 : (t > a.N ? a.N : t);  // non-finite logits must not produce a count outside 1..N
                     const size_t row = (size_t)bh * a.Cq + c0 + r;
                     a.t_c[row] = (int32_t)t;
                     a.rows[row].tau_key = tau;
@@ -622,13 +624,14 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
 
     // ordered emission
     uint32_t tk[R];
-    int nd[R];
+    int nd[R], cap[R];
     int64_t off[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         tk[r] = tau[r];
         nd[r] = need[r];
         off[r] = c0 + r < a.Cq ? a.key_offsets[(size_t)bh * a.Cq + c0 + r] : 0;
+        cap[r] = c0 + r < a.Cq ? a.r_c[(size_t)bh * a.Cq + c0 + r] : 0;  // the list's length: writes stay inside it
     }
     // With a code-count table the verdicts (above the threshold / in the threshold group, per row) are taken once
     // per distinct code and kept in the shared memory the descents no longer need; a key then looks its item up
@@ -730,12 +733,21 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
                 if (sl || ti) {
                     const int sb = wsel[r][q * NWARP + warp] + __popc(bs[q][r] & lt);
                     const int tb = wtie[r][q * NWARP + warp] + __popc(bt[q][r] & lt);
-                    if (sl || tb < nd[r])
-                        a.key_indices[off[r] + sb + min(tb, nd[r])] = j;
+                    const int slot = sb + min(tb, nd[r]);
+                    if ((sl || tb < nd[r]) && slot < cap[r])  // the second test only bites on non-finite logits
+                        a.key_indices[off[r] + slot] = j;
                 }
             }
         }
         __syncthreads();
+    }
+    // A list is always written in full (the counts are exact).  Only a plan over non-finite logits can fall short:
+    // its tail then gets key 0, so that whoever reads the list finds key indices and nothing else.
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int wrote = min(cap[r], base_sel[r] + min(base_tie[r], nd[r]));
+        for (int p = wrote + tid; p < cap[r]; p += NT)
+            a.key_indices[off[r] + p] = 0;
     }
 }
 

@@ -656,3 +656,42 @@ def test_concurrent_plans_on_many_streams():
         for dQ, dK, dV, plan, alone, out, stream in jobs:
             plan.check(f"repetition {rep}")
             assert torch.equal(out, alone)
+
+
+@pytest.mark.parametrize("what", ["nan_in_keys", "inf_in_queries", "all_nan"])
+def test_non_finite_inputs_neither_hang_nor_leave_the_buffers(what, monkeypatch):
+    """Inputs are assumed finite; with NaN / Inf in them the results are undefined, but every count stays in range,
+    every index written or read stays inside its buffer and the calls return.  Guard words around the index buffer
+    must be untouched, and the same plan object must give the exact plan again on clean inputs afterwards."""
+    cfg = inputs.CONFIGS["small"].replace(H=2)
+    Q, K, V = inputs.make_qkv(cfg, 81)
+    bad = [x.copy() for x in (Q, K, V)]
+    nan, inf = np.uint16(0x7FC0), np.uint16(0x7F80)
+    if what == "nan_in_keys":
+        bad[1][0, 0, 5::97, 3::11] = nan
+        bad[2][0, 1, 7, :] = nan
+    elif what == "inf_in_queries":
+        bad[0][0, :, 11::53, ::5] = inf
+        bad[1][0, 1, 100:140, 17] = np.uint16(0xFF80)  # -inf
+    else:
+        for x in bad:
+            x[:] = nan
+    plan = sb.Plan(sb.make_params(cfg))
+    # the index buffer ends the workspace; the binding's tensor is 256 bytes longer than the (256-byte aligned) workspace
+    assert plan.workspace.data_ptr() % 256 == 0
+    plan.workspace[-256:] = 0x5A
+    O = sb.scope_forward(_dev(bad[0]), _dev(bad[1]), _dev(bad[2]), plan)
+    torch.cuda.synchronize()
+    status, _ = plan.status()
+    assert status in (sb.SCOPE_OK, sb.SCOPE_ERR_CAPACITY)
+    assert bool((plan.workspace[-256:] == 0x5A).all())
+    for name in ("TOPP_COUNT", "BASE_COUNT", "FINAL_COUNT"):
+        v = plan.export(name)
+        assert v.min() >= 1 and v.max() <= cfg.N, name
+    assert plan.export("Q_ASSIGN").max() < cfg.Cq and plan.export("K_CODES_W").max() < cfg.Cw
+    # and the plan object is as good as new
+    plan.reset_status()
+    dQ, dK, dV = _dev(Q), _dev(K), _dev(V)
+    sb.scope_forward(dQ, dK, dV, plan)
+    plan.check()
+    _compare_plan(plan, _oracle_plans(Q, K, cfg), cfg)
