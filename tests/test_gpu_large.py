@@ -93,3 +93,39 @@ def test_full_size_layer_on_sampled_heads(name, heads):
         assert err <= 2e-2 and rel <= 1e-2, (name, h, err, rel)
         m_ref, t_ref, _ = orc.recall_rows(Q[0, h], K[0, h], g[h], Sg, cfg.scale, rrows[h], 0.1)
         assert np.array_equal(top[h], t_ref) and np.allclose(mass[h], m_ref, rtol=1e-11, atol=0), (name, h)
+
+
+def test_more_tokens_than_any_config():
+    """300 000 tokens per head (2.5x the largest configuration): structure that holds at any size, and attention
+    rows against the oracle given the CUDA path's own key sets (no full oracle plan at this size)."""
+    cfg = inputs.ScopeConfig("big", 1, 2, (50, 60, 100), (16, 56, 56), 128, 16, 64, 64, 3, 0.9, 512)
+    Q, K, V = inputs.make_qkv(cfg, seed=3, threads=16)
+    dQ, dK, dV = (sb.bits_to_torch(x, device="cuda") for x in (Q, K, V))
+    plan = sb.Plan(sb.make_params(cfg))
+    O = sb.scope_forward(dQ, dK, dV, plan)
+    plan.check()
+    O = O[0].float().cpu().numpy()
+    N, Cq = cfg.N, cfg.Cq
+    g, n_c = plan.export("Q_ASSIGN"), plan.export("CLUSTER_SIZES")
+    t_c, b_c, r_c, k_head = (plan.export(f) for f in ("TOPP_COUNT", "BASE_COUNT", "FINAL_COUNT", "K_HEAD"))
+    off, idx = plan.export("KEY_OFFSETS"), plan.export("KEY_INDICES")
+    perm, qoff = plan.export("Q_PERM"), plan.export("Q_OFFSETS")
+    assert np.array_equal(n_c.sum(1), np.full(cfg.H, N))
+    assert np.array_equal(b_c, np.maximum(t_c, cfg.k_fix))
+    for h in range(cfg.H):
+        assert np.array_equal(np.bincount(g[h], minlength=Cq), n_c[h])
+        assert k_head[h] == -(-int((n_c[h].astype(np.int64) * b_c[h]).sum()) // N)   # Eq. 9 in integers
+        assert np.array_equal(r_c[h], np.minimum(N, np.maximum(b_c[h], k_head[h])))
+        assert np.array_equal(np.sort(perm[h]), np.arange(N))
+        assert np.array_equal(g[h][perm[h]], np.repeat(np.arange(Cq), n_c[h]))
+    assert np.array_equal(np.diff(off), r_c.reshape(-1))
+    rng = np.random.default_rng(4)
+    for h in range(cfg.H):
+        Sg = [idx[off[h * Cq + c]: off[h * Cq + c + 1]] for c in range(Cq)]
+        for c in rng.choice(Cq, 8, replace=False):
+            assert np.all(np.diff(Sg[c]) > 0) and Sg[c][0] >= 0 and Sg[c][-1] < N   # ascending, distinct, in range
+        rows = rng.choice(N, 24, replace=False)
+        Oref = orc.attention_rows(Q[0, h], K[0, h], V[0, h], g[h], Sg, cfg.scale, rows)
+        err = np.abs(O[h][rows] - Oref).max()
+        rel = np.linalg.norm(O[h][rows] - Oref) / np.linalg.norm(Oref)
+        assert err <= 2e-2 and rel <= 1e-2, (h, err, rel)
