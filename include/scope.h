@@ -158,7 +158,9 @@ scope_status scope_plan_stages(const void *Q, const void *K, scope_plan_t *plan,
 scope_status scope_sparse_attn(const void *Q, const void *K, const void *V, const scope_plan_t *plan,
                                void *O, void *stream);
 
-/* scope_plan followed by scope_sparse_attn on the same stream. */
+/* scope_plan followed by scope_sparse_attn on the same stream.  Like them it only enqueues kernels and
+ * memsets on `stream`: plans on different streams run concurrently, and a stream capture records the
+ * call (make one call outside the capture first: function attributes and device queries are set then). */
 scope_status scope_forward(const void *Q, const void *K, const void *V, scope_plan_t *plan, void *O,
                            void *stream);
 

@@ -695,3 +695,29 @@ def test_non_finite_inputs_neither_hang_nor_leave_the_buffers(what, monkeypatch)
     sb.scope_forward(dQ, dK, dV, plan)
     plan.check()
     _compare_plan(plan, _oracle_plans(Q, K, cfg), cfg)
+
+
+def test_layer_can_be_captured_into_a_cuda_graph():
+    """scope_forward only enqueues kernels and memsets on the given stream (no allocation, no synchronisation), so a
+    stream capture records it; replays give the eager result, also after the inputs changed in place."""
+    cfg = inputs.CONFIGS["small"].replace(H=3)
+    Q, K, V, dQ, dK, dV = _layer(cfg, 91)
+    plan = sb.Plan(sb.make_params(cfg))
+    O = torch.empty_like(dQ)
+    sb.scope_forward(dQ, dK, dV, plan, O)   # first call outside the capture (function attributes, one-time queries)
+    plan.check()
+    eager = O.clone()
+    graph = torch.cuda.CUDAGraph()
+    O.zero_()
+    with torch.cuda.graph(graph):
+        sb.scope_forward(dQ, dK, dV, plan, O)
+    graph.replay()
+    torch.cuda.synchronize()
+    plan.check()
+    assert torch.equal(O, eager)
+    Q2, K2, V2 = inputs.make_qkv(cfg, 92)
+    dQ.copy_(_dev(Q2)); dK.copy_(_dev(K2)); dV.copy_(_dev(V2))
+    graph.replay()
+    torch.cuda.synchronize()
+    plan.check()
+    _compare_plan(plan, _oracle_plans(Q2, K2, cfg), cfg)
