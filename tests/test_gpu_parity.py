@@ -721,3 +721,46 @@ def test_layer_can_be_captured_into_a_cuda_graph():
     torch.cuda.synchronize()
     plan.check()
     _compare_plan(plan, _oracle_plans(Q2, K2, cfg), cfg)
+
+
+@pytest.mark.parametrize("case", ["coarse_tables", "two_values", "negative_zero", "wide_range"])
+@pytest.mark.parametrize("mode,mname", [(sb.SELECT_ONLINE, "online"), (sb.SELECT_TOPP, "topp")])
+def test_selection_on_crafted_tables_with_many_ties(case, mode, mname):
+    """The selection stage alone, fed tables and codes made to tie: logits on a coarse grid (thousands of keys per
+    value, thresholds that fall inside a tie group), two-valued rows, rows of +0 / -0, and a range of 1e6.  Counts and
+    key sets must equal the oracle's exactly (ties go to the lower key index)."""
+    cfg = inputs.CONFIGS["small"].replace(H=2, top_p=0.83, k_fix=37)
+    rng = np.random.default_rng({"coarse_tables": 1, "two_values": 2, "negative_zero": 3, "wide_range": 4}[case])
+    N, Cq, Cs = cfg.N, cfg.Cq, (cfg.Ct, cfg.Ch, cfg.Cw)
+    plan = sb.Plan(sb.make_params(cfg, index_capacity=cfg.H * Cq * N, select_mode=mode))
+    P, z, n_c = [], [], []
+    for h in range(cfg.H):
+        if case == "coarse_tables":
+            tabs = [rng.integers(-3, 4, (Cq, c)).astype(np.float32) * 0.5 for c in Cs]
+        elif case == "two_values":
+            tabs = [np.where(rng.random((Cq, c)) < 0.3, 1.0, 0.0).astype(np.float32) for c in Cs]
+        elif case == "negative_zero":
+            tabs = [np.where(rng.random((Cq, c)) < 0.5, 0.0, -0.0).astype(np.float32) for c in Cs]
+            tabs[0][::3] = rng.integers(-1, 2, tabs[0][::3].shape).astype(np.float32)
+        else:
+            tabs = [(rng.standard_normal((Cq, c)) * 10.0 ** rng.integers(-3, 4, (Cq, 1))).astype(np.float32) for c in Cs]
+        P.append(tabs)
+        z.append([rng.integers(0, c, N).astype(np.int32) for c in Cs])
+        sizes = rng.multinomial(N, np.ones(Cq) / Cq).astype(np.int32)
+        sizes[0] += sizes[1]
+        sizes[1] = 0  # an empty query cluster
+        n_c.append(sizes)
+    for m, nm in enumerate("THW"):
+        plan.import_(f"LUT_{nm}", np.stack([P[h][m] for h in range(cfg.H)]))
+        plan.import_(f"K_CODES_{nm}", np.stack([z[h][m] for h in range(cfg.H)]))
+    plan.import_("CLUSTER_SIZES", np.stack(n_c))
+    sb.scope_plan_stages(None, None, plan, sb.STAGE_SELECT)
+    plan.check()
+    t_c, b_c, r_c, k_head = (plan.export(f) for f in ("TOPP_COUNT", "BASE_COUNT", "FINAL_COUNT", "K_HEAD"))
+    for h in range(cfg.H):
+        t, b, k, r, S, margin = orc.select_head(tuple(P[h]), tuple(z[h]), n_c[h], N, cfg.scale, cfg.top_p, cfg.k_fix, mname)
+        assert np.array_equal(t_c[h], t), (case, h, np.nonzero(t_c[h] != t)[0][:5])
+        assert np.array_equal(b_c[h], b) and k_head[h] == k and np.array_equal(r_c[h], r)
+        got = _key_sets(plan, h, Cq)
+        for c in range(Cq):
+            assert np.array_equal(got[c], S[c]), (case, h, c)
