@@ -551,3 +551,40 @@ def test_partitions_into_more_ranges(M):
     three = orc.scores_row_m([P[c] for P in pl.P[:3]], pl.z[:3])
     assert np.array_equal(three, orc.scores_row(pl.P[0][c], pl.P[1][c], pl.P[2][c], *pl.z[:3]))
     assert all(s.shape[0] == r for s, r in zip(pl.S, pl.r_c)) and np.all(pl.r_c >= pl.k_head)
+
+
+# ----------------------------------------------------------------------------- randomised invariants of Algorithm 3
+
+
+def _random_selection_case(rng, N, Cq, Cs, grid):
+    P = tuple((rng.integers(-grid, grid + 1, (Cq, c)) / 2.0).astype(np.float32) for c in Cs)
+    z = tuple(rng.integers(0, c, N).astype(np.int32) for c in Cs)
+    n_c = rng.multinomial(N, rng.dirichlet(np.ones(Cq))).astype(np.int32)
+    return P, z, n_c
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_selection_invariants_on_random_tied_tables(seed):
+    """Algorithm 3 on random tables whose entries sit on a coarse grid (so that logits tie by the hundred): every
+    property that Eq. 7 - Eq. 10 fix without reference to an implementation."""
+    rng = np.random.default_rng(seed)
+    N, Cq, Cs = int(rng.integers(40, 400)), int(rng.integers(1, 9)), tuple(int(v) for v in rng.integers(1, 7, 3))
+    rho, k_fix = float(rng.choice([0.3, 0.5, 0.9, 0.97])), int(rng.integers(1, N + 1))
+    P, z, n_c = _random_selection_case(rng, N, Cq, Cs, int(rng.integers(1, 4)))
+    scale = 0.37
+    t, b, k, r, S, _ = orc.select_head(P, z, n_c, N, scale, rho, k_fix)
+    assert np.array_equal(b, np.maximum(t, k_fix))                                   # Eq. 8
+    assert k == -(-int((n_c.astype(np.int64) * b).sum()) // N)                       # Eq. 9, exact ceiling
+    assert np.array_equal(r, np.minimum(N, np.maximum(b, k)))                        # Eq. 10
+    for c in range(Cq):
+        raw = (P[0][c][z[0]] + P[1][c][z[1]]) + P[2][c][z[2]]
+        s = raw.astype(np.float64) * float(np.float32(scale))
+        a = np.exp(s - s.max())
+        a /= a.sum()
+        order = np.lexsort((np.arange(N), -raw))                                      # descending logit, then key index
+        cum = np.cumsum(a[order])
+        assert cum[t[c] - 1] >= rho - 1e-12 and (t[c] == 1 or cum[t[c] - 2] < rho + 1e-12)   # Eq. 7: smallest prefix
+        assert np.array_equal(S[c], np.sort(order[:r[c]]))                            # the first r_c of the ranking
+    # more mass or a higher floor never removes a key
+    t2, b2, k2, r2, S2, _ = orc.select_head(P, z, n_c, N, scale, min(1.0, rho + 0.02), min(N, k_fix + 3))
+    assert all(np.isin(S[c], S2[c]).all() for c in range(Cq))
