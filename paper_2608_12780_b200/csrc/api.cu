@@ -423,7 +423,7 @@ static scope_status run_stages(const void *Q, const void *K, scope_plan_t *pl, u
     const scope_params &p = pl->p;
 
     if (stages & SCOPE_STAGE_SELECT) {
-        // a fresh selection clears an earlier capacity verdict
+        // a fresh selection clears an earlier capacity error
         if (cudaMemsetAsync(pl->status, 0, ST_WORDS * sizeof(int32_t), st) != cudaSuccess)
             return SCOPE_ERR_CUDA;
     }

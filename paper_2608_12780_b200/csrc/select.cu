@@ -633,10 +633,10 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
         off[r] = c0 + r < a.Cq ? a.key_offsets[(size_t)bh * a.Cq + c0 + r] : 0;
         cap[r] = c0 + r < a.Cq ? a.r_c[(size_t)bh * a.Cq + c0 + r] : 0;  // the list's length: writes stay inside it
     }
-    // With a code-count table the verdicts (above the threshold / in the threshold group, per row) are taken once
+    // With a code-count table the marks (above the threshold / in the threshold group, per row) are set once
     // per distinct code and kept in the shared memory the descents no longer need; a key then looks its item up
     // through its cell instead of evaluating four proxy logits.
-    uint8_t *verdict = reinterpret_cast<uint8_t *>(cnt);
+    uint8_t *mark = reinterpret_cast<uint8_t *>(cnt);
     const bool by_item = !WIDE && a.cells > 0 && nitems <= R * NB * (int)sizeof(uint32_t);
     const int32_t *cell_item = a.cell_table + (size_t)bh * a.cells;
     if (by_item) {
@@ -651,7 +651,7 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
                 v |= (key > tk[r] ? 1u : 0u) << r;
                 v |= (key == tk[r] ? 1u : 0u) << (R + r);
             }
-            verdict[i] = (uint8_t)v;
+            mark[i] = (uint8_t)v;
         }
         __syncthreads();
     }
@@ -671,13 +671,13 @@ __global__ void __launch_bounds__(NT, 2) select_emit_kernel(SelectArgs a)
                 item[q] = j0 + q * NT + tid < a.N ? __ldg(cell_item + code_cell(code[q], a.Ch, a.Cw)) : 0;
         }
         uint32_t bs[SUB][R], bt[SUB][R];
-        uint32_t mine = 0u;  // this thread's verdicts: sub-chunk q in byte q (bit r: above, bit R + r: threshold group)
+        uint32_t mine = 0u;  // this thread's marks: sub-chunk q in byte q (bit r: above, bit R + r: threshold group)
 #pragma unroll
         for (int q = 0; q < SUB; ++q) {
             const int j = j0 + q * NT + tid;
             uint32_t v = 0u;
             if (j < a.N && by_item) {
-                v = verdict[item[q]];
+                v = mark[item[q]];
             } else if (j < a.N) {
                 const ExtraCodes xc = extra_codes<WIDE>(a, bh, j);
 #pragma unroll
