@@ -81,24 +81,26 @@ struct GroupShared {
     uint64_t mbar;
 };
 
-__device__ __forceinline__ void load_x_tile(const KmArgs &a, const bf16 *Xh, int tok0, uint32_t xbase, int gt)
+__device__ __forceinline__ void load_x_tile(const KmArgs &a, const bf16 *Xh, int tok0, uint32_t xbase, int gt, int pt)
 {
     // 128 rows x 16 chunks of 16 bytes; rows past N are zero.  A thread keeps its chunk and walks rows
-    // gt/16 + 8 i: the swizzle term depends on row & 7 only, so the destination advances by 1024 bytes.
-    const int row0 = gt >> 4, chunk = gt & 15;
+    // gt/16 + rs i (rs = 8 rows for a pipeline of 128 threads, 16 for one of 256): the swizzle term depends on
+    // row & 7 only, so the destination advances by rs x 128 bytes.
+    const int row0 = gt >> 4, chunk = gt & 15, rs = pt >> 4;
     const uint32_t dst = xbase + (chunk >> 3) * HALF_BYTES + sw128(row0, chunk & 7);
     const bf16 *src = Xh + (int64_t)(tok0 + row0) * a.sn + chunk * 8;
-    const int64_t step = 8 * a.sn;
-    const int rows_left = a.N - tok0 - row0;  // row row0 + 8 i exists iff 8 i < rows_left
-#pragma unroll
-    for (int i = 0; i < TM / 8; ++i) {
-        const bool ok = 8 * i < rows_left;
-        cp_async16_zfill(dst + 1024 * i, ok ? src : Xh, ok ? 16 : 0);
+    const int64_t step = (int64_t)rs * a.sn;
+    const int rows_left = a.N - tok0 - row0;  // row row0 + rs i exists iff rs i < rows_left
+#pragma unroll 8
+    for (int i = 0; i < TM / rs; ++i) {
+        const bool ok = rs * i < rows_left;
+        cp_async16_zfill(dst + rs * 128 * i, ok ? src : Xh, ok ? 16 : 0);
         src += step;
     }
     cp_async_commit();
 }
 
+template <bool WIDE>
 __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int tiles_per_block, int groups, int32_t *status)
 {
     extern __shared__ unsigned char smem_dyn[];
@@ -115,8 +117,15 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
     __shared__ int s_queue;  // next tile of the block's range nobody has taken yet
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int grp = tid >> 7, gt = tid & 127;       // pipeline, thread within it
-    const int gw = warp & 3;                        // warp within the pipeline = TMEM lane quarter
+    // A pipeline is 128 threads, one per token of its tile.  A block that has room for one pipeline only (large
+    // codebooks) runs it 256 wide: the second 128 threads help with the copies, scan the upper half of every
+    // range's columns for the same tokens and take their share of the member sums.
+    constexpr bool wide = WIDE;
+    constexpr int pt = WIDE ? 256 : 128;
+    const int grp = wide ? 0 : tid >> 7, gt = wide ? tid : tid & 127;  // pipeline, thread within it
+    const int tk = gt & 127;                        // the thread's token (row of the tile, TMEM lane)
+    const bool helper = WIDE && gt >= 128;
+    const int gw = warp & 3;                        // TMEM lane quarter of the warp
     const int bh = blockIdx.y;
     const int b = bh / a.H, h = bh % a.H;
     const bf16 *Xh = a.X + (int64_t)b * a.sb + (int64_t)h * a.sh;
@@ -168,8 +177,8 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
     // the pipelines of a block share one queue over the block's tiles: whichever is free takes the next tile
     for (int tile = first; tile < last && !dead; tile = G.next_tile) {
         const int tok0 = tile * TM;
-        const bool valid = tok0 + gt < a.N;
-        load_x_tile(a, Xh, tok0, xbase, gt);
+        const bool valid = tok0 + tk < a.N;
+        load_x_tile(a, Xh, tok0, xbase, gt, pt);
         cp_async_wait<0>();
         if (a.rope.on && !a.x2_ready) {
             // First pass over a tensor that still lacks its rotary embedding: every thread rotates the 16-byte
@@ -189,26 +198,26 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             }
             unsigned char *px = s_x + grp * XTILE_BYTES + (chunk >> 3) * HALF_BYTES + sw128(row0, chunk & 7);
             bf16 *gx = a.Xw + (int64_t)b * a.sb + (int64_t)h * a.sh + (int64_t)(tok0 + row0) * a.sn + chunk * 8;
-            const int plane = a.rope.Hg * a.rope.Wg;
-            for (int i = 0; i < TM / 8 && tok0 + row0 + 8 * i < a.N; ++i) {
-                const int n = tok0 + row0 + 8 * i;
-                const int pt = n / plane, rem = n - pt * plane, ph = rem / a.rope.Wg, pw = rem - ph * a.rope.Wg;
-                uint4 v = *reinterpret_cast<uint4 *>(px + 1024 * i);
+            const int plane = a.rope.Hg * a.rope.Wg, rs = pt >> 4;
+            for (int i = 0; i < TM / rs && tok0 + row0 + rs * i < a.N; ++i) {
+                const int n = tok0 + row0 + rs * i;
+                const int p_t = n / plane, rem = n - p_t * plane, ph = rem / a.rope.Wg, pw = rem - ph * a.rope.Wg;
+                uint4 v = *reinterpret_cast<uint4 *>(px + rs * 128 * i);
                 uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const int pos = axis[q] == 0 ? pt : (axis[q] == 1 ? ph : pw);
+                    const int pos = axis[q] == 0 ? p_t : (axis[q] == 1 ? ph : pw);
                     const size_t at = (size_t)pos * half[q] + idx[q];
                     w[q] = rope_word(w[q], __ldg(a.rope.cs[axis[q]] + at), __ldg(a.rope.sn[axis[q]] + at));
                 }
                 v = make_uint4(w[0], w[1], w[2], w[3]);
-                *reinterpret_cast<uint4 *>(px + 1024 * i) = v;
-                *reinterpret_cast<uint4 *>(gx + (int64_t)8 * i * a.sn) = v;
+                *reinterpret_cast<uint4 *>(px + rs * 128 * i) = v;
+                *reinterpret_cast<uint4 *>(gx + (int64_t)rs * i * a.sn) = v;
             }
         }
         fence_proxy_async();
         tc_fence_before();
-        bar_sync(1 + grp, 128);
+        bar_sync(1 + grp, pt);
         // ---- distances on the tensor core: one thread issues, the others take the row norms meanwhile
         if (gt == 0) {
             tc_fence_after();
@@ -235,26 +244,26 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             }
             mma_commit(&G.mbar);
         }
-        for (int e = gt; e < MAXC_ALL / 4; e += 128)
+        for (int e = gt; e < MAXC_ALL / 4; e += pt)
             G.cnt[e] = 0u;
         // squared norm of the whole row (an upper bound of every range's slice, used in the tolerance): taken
         // from the tile in the first pass of a call and kept in global memory for the later ones
         // the label word of the pass before (incremental passes compare against it): asked for early, used late
         uint32_t old_word = 0u;
-        if (a.incremental && valid) {
-            const size_t at = (size_t)bh * a.N + tok0 + gt;
+        if (a.incremental && valid && !helper) {
+            const size_t at = (size_t)bh * a.N + tok0 + tk;
             old_word = a.single_field > 0 ? __ldg(a.codes + (size_t)((a.single_field - 1) / 3) * a.B * a.H * a.N + at)
                                           : (a.nspaces == 1 ? (uint32_t)__ldg(a.assign + at) : __ldg(a.codes + at));
         }
         float x2 = 0.f;
         if (a.x2 != nullptr && a.x2_ready) {
-            if (valid)
-                x2 = __ldg(a.x2 + (size_t)bh * a.N + tok0 + gt);
-        } else {
+            if (valid && !helper)
+                x2 = __ldg(a.x2 + (size_t)bh * a.N + tok0 + tk);
+        } else if (!helper) {
             float x2a = 0.f, x2b = 0.f;
 #pragma unroll
             for (int chunk = 0; chunk < 16; ++chunk) {
-                uint4 raw = *reinterpret_cast<const uint4 *>(s_x + grp * XTILE_BYTES + (chunk >> 3) * HALF_BYTES + sw128(gt, chunk & 7));
+                uint4 raw = *reinterpret_cast<const uint4 *>(s_x + grp * XTILE_BYTES + (chunk >> 3) * HALF_BYTES + sw128(tk, chunk & 7));
                 const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
@@ -265,7 +274,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             }
             x2 = x2a + x2b;
             if (a.x2 != nullptr && valid)
-                a.x2[(size_t)bh * a.N + tok0 + gt] = x2;
+                a.x2[(size_t)bh * a.N + tok0 + tk] = x2;
         }
         // a wait that runs out is recorded and ends this pipeline after the next barrier
         const bool ok = __all_sync(0xffffffffu, mbar_wait(&G.mbar, phase));
@@ -275,17 +284,22 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         }
         phase ^= 1;
         tc_fence_after();
-        if (ok) {
-            for (int s = 0; s < a.nspaces; ++s) {
-                const int C = a.sp[s].C, cp = L.cpad[s];
-                const float *un = s_un + L.un_off[s];
-                const uint32_t ta = tmem_g + ((uint32_t)(gw * 32) << 16) + L.col[s];
+        for (int s = 0; s < a.nspaces; ++s) {
+            const int C = a.sp[s].C, cp = L.cpad[s];
+            const float *un = s_un + L.un_off[s];
+            const uint32_t ta = tmem_g + ((uint32_t)(gw * 32) << 16) + L.col[s];
+            // a 256-wide pipeline splits the columns of the (single) range between a token's two threads
+            const int csplit = wide ? min(cp, (cp / 2 + 31) & ~31) : cp;
+            const int c_lo = helper ? csplit : 0, c_hi = helper ? cp : csplit;
+            float best = INFINITY, second = INFINITY;
+            int arg = 0;
+            if (ok) {
                 // four independent running (best, second, index) triples over the columns j % 4, merged at the
                 // end: the chain of dependent compares is what this loop waits on.  Which of several equal
                 // distances wins here does not matter: a zero gap is always a close call.
                 float bq[4] = {INFINITY, INFINITY, INFINITY, INFINITY}, sq[4] = {INFINITY, INFINITY, INFINITY, INFINITY};
                 int aq[4] = {0, 0, 0, 0};
-                for (int c0 = 0; c0 < cp; c0 += 32) {
+                for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
                     uint32_t r[32];
                     if (cp - c0 >= 32) {
                         tmem_ld32(ta + c0, r);
@@ -315,15 +329,34 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                         }
                     }
                 }
-                float best = bq[0], second = sq[0];
-                int arg = aq[0];
+                best = bq[0];
+                second = sq[0];
+                arg = aq[0];
 #pragma unroll
                 for (int q = 1; q < 4; ++q) {
                     second = fminf(fminf(second, sq[q]), fmaxf(best, bq[q]));
                     arg = bq[q] < best ? aq[q] : arg;
                     best = fminf(best, bq[q]);
                 }
-                G.asg[s][gt] = (uint16_t)arg;
+            }
+            if (wide) {
+                // the helper hands its (best, second, index) to the token's owner through the run list's storage,
+                // which nothing uses before the labels are out (a 256-wide pipeline has one range)
+                if (helper) {
+                    G.runs[0][tk] = __float_as_uint(best);
+                    G.runs[1][tk] = __float_as_uint(second);
+                    G.runs[2][tk] = (uint32_t)arg;
+                }
+                bar_sync(1 + grp, pt);
+                if (!helper) {
+                    const float hb = __uint_as_float(G.runs[0][tk]), hs = __uint_as_float(G.runs[1][tk]);
+                    second = fminf(fminf(second, hs), fmaxf(best, hb));
+                    arg = hb < best ? (int)G.runs[2][tk] : arg;
+                    best = fminf(best, hb);
+                }
+            }
+            if (ok && !helper) {
+                G.asg[s][tk] = (uint16_t)arg;
                 const int cbeg = a.sp[s].ch0 & ~15, cend = (a.sp[s].ch0 + a.sp[s].D + 15) & ~15;
                 // error budget of two tensor-core evaluations of |u|^2 - 2 x.u: the products are exact, each of
                 // the NSPLIT * (channels / 16) accumulating MMAs may lose up to two fp32 ulps of the running
@@ -372,20 +405,20 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                             base = atomicAdd(&G.ncand, nc);
                         if (base + nc <= MAXCAND) {
                             for (int k = 0; k < nc; ++k)
-                                G.cand[base + k] = (uint32_t)((packed >> (16 * k)) & 0x3ffu) | ((uint32_t)gt << 10) | ((uint32_t)s << 17) |
+                                G.cand[base + k] = (uint32_t)((packed >> (16 * k)) & 0x3ffu) | ((uint32_t)tk << 10) | ((uint32_t)s << 17) |
                                                    ((uint32_t)k << 19) | ((uint32_t)nc << 21);
                         } else {  // many contenders (or a full list): every centroid is re-evaluated
                             for (int k = base; k < MAXCAND; ++k)
                                 G.cand[k] = 1u << 19;  // reserved but unused slots: never the first of a token
                             int slot = atomicAdd(&G.nflagged, 1);
-                            G.flagged[slot] = (uint16_t)((s << 8) | gt);
+                            G.flagged[slot] = (uint16_t)((s << 8) | tk);
                         }
                     }
                 }
             }
         }
         tc_fence_before();
-        bar_sync(1 + grp, 128);
+        bar_sync(1 + grp, pt);
         dead = *reinterpret_cast<volatile int *>(&G.dead) != 0;
         if (dead)
             break;
@@ -413,7 +446,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                     }
                     G.cdist[gt] = d;
                 }
-                bar_sync(1 + grp, 128);
+                bar_sync(1 + grp, pt);
                 if (gt < ncand) {
                     const uint32_t e = G.cand[gt];
                     if (((e >> 19) & 3) == 0) {  // first contender of its token: ascending centroid order, lowest wins ties
@@ -430,7 +463,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                 }
             }
             const int nf = G.nflagged;
-            for (int f = gw; f < nf; f += 4) {
+            for (int f = gt >> 5; f < nf; f += pt >> 5) {
                 const int s = G.flagged[f] >> 8, lt = G.flagged[f] & 0xff;
                 const KmSpace &sp = a.sp[s];
                 const float *cent = sp.cent + (size_t)bh * sp.C * sp.D;
@@ -470,15 +503,15 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                     G.asg[s][lt] = (uint16_t)ba;
             }
         }
-        bar_sync(1 + grp, 128);
+        bar_sync(1 + grp, pt);
 
         // ---- labels out.  A full pass groups the tile's tokens by label (counting sort in shared memory) and sums
         // the members of every label present; an incremental pass lists the tokens whose label changed.
         int lab[3] = {0, 0, 0}, pos[3] = {0, 0, 0};
-        if (valid) {
-            const size_t at = (size_t)bh * a.N + tok0 + gt;
+        if (valid && !helper) {
+            const size_t at = (size_t)bh * a.N + tok0 + tk;
             for (int s = 0; s < a.nspaces; ++s)
-                lab[s] = G.asg[s][gt];
+                lab[s] = G.asg[s][tk];
             int old[3] = {lab[0], lab[1], lab[2]};
             if (a.single_field > 0) {
                 // one range of the keys per launch (T, then H, then W, ...): three 10-bit fields a word; word w of all
@@ -502,7 +535,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             for (int s = 0; s < a.nspaces; ++s) {
                 if (a.incremental) {
                     if (old[s] != lab[s])  // token | old label << 7 | new label << 17
-                        G.runs[s][atomicAdd(&G.nruns[s], 1)] = (uint32_t)gt | ((uint32_t)old[s] << 7) | ((uint32_t)lab[s] << 17);
+                        G.runs[s][atomicAdd(&G.nruns[s], 1)] = (uint32_t)tk | ((uint32_t)old[s] << 7) | ((uint32_t)lab[s] << 17);
                 } else {
                     const int sh = (lab[s] & 3) * 8;
                     pos[s] = (int)((atomicAdd(&G.cnt[(L.un_off[s] + lab[s]) >> 2], 1u << sh) >> sh) & 0xffu);
@@ -510,7 +543,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             }
         }
         if (a.incremental) {
-            bar_sync(1 + grp, 128);
+            bar_sync(1 + grp, pt);
             // member totals follow the moved tokens: + x to the new label, - x to the old one (fp64 sums of bf16
             // values are exact, so the totals equal a fresh summation); a thread owns two adjacent channels
             const int ch = 2 * (gt & 63), hf = gt >> 6;
@@ -525,7 +558,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                 const uint32_t xpair = xbase + (ch >> 6) * HALF_BYTES + (ch & 7) * 2;
                 const uint32_t cbits = (uint32_t)((ch & 63) >> 3) << 4;
                 const int nm = G.nruns[s];
-                for (int e = hf; e < nm; e += 2) {
+                for (int e = hf; e < nm; e += pt >> 6) {
                     const uint32_t mv = G.runs[s][e];
                     const int lt = mv & 127, from = (mv >> 7) & 1023, to = mv >> 17;
                     const uint32_t w = lds32(xpair + (sw128(lt, 0) ^ cbits));
@@ -543,13 +576,13 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             if (gt == 0)
                 G.next_tile = atomicAdd(&s_queue, 1);
             tc_fence_before();
-            bar_sync(1 + grp, 128);  // the X tile and the label arrays are reused by the next tile
+            bar_sync(1 + grp, pt);  // the X tile and the label arrays are reused by the next tile
             continue;
         }
-        bar_sync(1 + grp, 128);
-        if (gw < a.nspaces) {
+        bar_sync(1 + grp, pt);
+        if ((gt >> 5) < a.nspaces) {
             // one warp per range: exclusive scan of the counts, list of the non-empty labels
-            const int s = gw, cp = L.cpad[s];
+            const int s = gt >> 5, cp = L.cpad[s];
             int base = 0, nr = 0;
             for (int c0 = 0; c0 < cp; c0 += 32) {
                 const int c = c0 + lane;
@@ -573,11 +606,11 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             if (lane == 0)
                 G.nruns[s] = nr;
         }
-        bar_sync(1 + grp, 128);
-        if (valid)
+        bar_sync(1 + grp, pt);
+        if (valid && !helper)
             for (int s = 0; s < a.nspaces; ++s)
-                G.sorted[s][G.start[L.un_off[s] + lab[s]] + pos[s]] = (uint16_t)sw128(gt, 0);
-        bar_sync(1 + grp, 128);
+                G.sorted[s][G.start[L.un_off[s] + lab[s]] + pos[s]] = (uint16_t)sw128(tk, 0);
+        bar_sync(1 + grp, pt);
 
         // ---- member sums: a thread owns two adjacent channels (one 32-bit word of every row) and every other
         // run of their range; one fp64 atomic per (label present in the tile, channel)
@@ -594,7 +627,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
             const uint32_t xpair = xbase + (ch >> 6) * HALF_BYTES + (ch & 7) * 2;
             const uint32_t cbits = (uint32_t)((ch & 63) >> 3) << 4;
             const int nr = (rel >= 0 && rel < sp.D) ? G.nruns[s] : 0;  // a one-range launch leaves the other channels alone
-            for (int r = hf; r < nr; r += 2) {
+            for (int r = hf; r < nr; r += pt >> 6) {
                 const uint32_t run = G.runs[s][r];
                 const int cl = run & 1023, st = (run >> 10) & 255, n = run >> 18;
                 const uint16_t *tok = &G.sorted[s][st];
@@ -625,7 +658,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         if (gt == 0)
             G.next_tile = atomicAdd(&s_queue, 1);
         tc_fence_before();
-        bar_sync(1 + grp, 128);  // the X tile and the label arrays are reused by the next tile
+        bar_sync(1 + grp, pt);  // the X tile and the label arrays are reused by the next tile
     }
 
     cp_async_wait<0>();
@@ -673,7 +706,10 @@ void launch_kmeans_assign_tc(const KmArgs &a, int32_t *status, cudaStream_t st)
     // a block must own its SM (it allocates all 512 TMEM columns): ask for more than half the shared memory
     if (smem < 120 * 1024)
         smem = 120 * 1024;
-    cudaFuncSetAttribute(kmeans_assign_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // a lone pipeline over one range (codebooks of a few hundred centroids) runs 256 threads wide
+    const bool wide = groups == 1 && a.nspaces == 1;
+    auto kernel = wide ? kmeans_assign_tc_kernel<true> : kmeans_assign_tc_kernel<false>;
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     const int ntiles = (a.N + TM - 1) / TM;
     // Blocks per head: a block pays for loading the codebook and ends when its slowest pipeline does, so few
     // large blocks are better, as long as the grid fills whole waves of SMs.  Cost model: waves x (rounds of
@@ -702,7 +738,7 @@ void launch_kmeans_assign_tc(const KmArgs &a, int32_t *status, cudaStream_t st)
     }
     const int tiles_per_block = (ntiles + best_bph - 1) / best_bph;
     dim3 grid((ntiles + tiles_per_block - 1) / tiles_per_block, heads);
-    kmeans_assign_tc_kernel<<<grid, 128 * groups, smem, st>>>(a, tiles_per_block, groups, status);
+    kernel<<<grid, wide ? 256 : 128 * groups, smem, st>>>(a, tiles_per_block, groups, status);
     count_launch();
 }
 
