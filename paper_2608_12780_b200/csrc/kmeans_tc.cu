@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
     }
     if (gt == 0) {
         G.dead = 0;
-        mbar_init(&G.mbar, 1);
+        mbar_init(&G.mbar, WIDE ? 2 : 1);
         mbar_fence_init();
     }
     // codebook splits and norms -> shared memory (once per block)
@@ -218,20 +218,26 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
         fence_proxy_async();
         tc_fence_before();
         bar_sync(1 + grp, pt);
-        // ---- distances on the tensor core: one thread issues, the others take the row norms meanwhile
+        // ---- distances on the tensor core: one thread issues, the others take the row norms meanwhile.  In a
+        // 256-wide pipeline the first thread of either half issues the columns its half will scan: two column
+        // blocks, two issuing threads (one thread issues at most one instruction per ~100 cycles).
         if (gt == 0) {
-            tc_fence_after();
             G.nflagged = 0;
             G.ncand = 0;
             if (a.incremental)
                 G.nruns[0] = G.nruns[1] = G.nruns[2] = 0;  // moved tokens per range
+        }
+        if (tk == 0) {
+            tc_fence_after();
             for (int s = 0; s < a.nspaces; ++s) {
                 const int cp = L.cpad[s];
                 const int k_lo = a.sp[s].ch0 >> 4, k_hi = (a.sp[s].ch0 + a.sp[s].D + 15) >> 4;
                 const uint32_t cb = smem_u32(s_cent) + L.cent_off[s];
-                // one instruction covers up to 256 centroids: larger codebooks take two column blocks
-                for (int n0 = 0; n0 < cp; n0 += 256) {
-                    const uint32_t idesc = idesc_bf16(TM, min(256, cp - n0), false, false);
+                const int csplit = wide ? min(cp, (cp / 2 + 31) & ~31) : cp;
+                const int n_lo = helper ? csplit : 0, n_hi = helper ? cp : csplit;
+                // one instruction covers up to 256 centroids: larger blocks take two
+                for (int n0 = n_lo; n0 < n_hi; n0 += 256) {
+                    const uint32_t idesc = idesc_bf16(TM, min(256, n_hi - n0), false, false);
                     bool acc = false;
                     for (int p = 0; p < NSPLIT; ++p)
                         for (int ks = k_lo; ks < k_hi; ++ks) {
@@ -242,7 +248,7 @@ __global__ void __launch_bounds__(NT, 1) kmeans_assign_tc_kernel(KmArgs a, int t
                         }
                 }
             }
-            mma_commit(&G.mbar);
+            mma_commit(&G.mbar);  // the barrier counts one arrival per issuing thread
         }
         for (int e = gt; e < MAXC_ALL / 4; e += pt)
             G.cnt[e] = 0u;
